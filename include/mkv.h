@@ -1,0 +1,194 @@
+/*
+ * mkv -- Moment-KV decode hot path for NVIDIA B200 (sm_100a), C ABI.
+ *
+ * One context holds, for `layers` attention layers and `batch` sequences, the
+ * frozen prefill K/V pool, the budget-bounded decode K/V pool, one importance
+ * score and one position id per decode-pool token.  mkv_decode_step() performs,
+ * for one layer and all sequences, one pass of Algorithm 1 of the Moment-KV
+ * paper (Sec. 4.2) minus the Q/K/V projection: append, attention over prefill U
+ * decode pool, head mean, momentum update of the importance, lowest-score
+ * eviction and in-place compaction.  Everything runs in CUDA kernels on the
+ * caller's stream; there is no CPU fallback.
+ *
+ * Conventions (all entry points)
+ *   - Return value: mkv_status.  No exceptions, no abort, no device trap.
+ *   - "device pointer": memory of the context's GPU, owned by the caller, only
+ *     read/written during the call's kernels (stream order); never retained.
+ *   - "host pointer": ordinary host memory, read/written before return unless
+ *     stated otherwise.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = legacy default stream).
+ *   - The library allocates NO device memory: the caller passes one workspace of
+ *     mkv_workspace_bytes() bytes, 256-byte aligned, which must outlive the
+ *     context.  mkv_destroy() frees host state only.
+ *   - Tensor layouts are row-major with the last index contiguous.
+ *     q, out: [batch][q_heads][head_dim]; k_new, v_new: [batch][kv_heads][head_dim].
+ *   - Query head h reads KV head h / (q_heads / kv_heads).
+ *   - Errors found on the host are returned at once; errors found by a kernel
+ *     (a count beyond capacity, a bounded wait that expired) set a sticky device
+ *     status word that mkv_status_sync() reads.
+ *   - One host thread at a time per context.
+ */
+#ifndef MKV_H_
+#define MKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mkv_ctx mkv_ctx; /* opaque, host-owned */
+
+typedef enum {
+    MKV_OK = 0,
+    MKV_ERR_INVALID_ARG = 1,  /* NULL pointer, value out of range                     */
+    MKV_ERR_BAD_STATE = 2,    /* e.g. decode step on a layer that was never prefilled */
+    MKV_ERR_CAPACITY = 3,     /* prefill longer than max_prefill, budget above create */
+    MKV_ERR_WORKSPACE = 4,    /* workspace too small or misaligned                    */
+    MKV_ERR_UNSUPPORTED = 5,  /* shape/dtype combination without a kernel             */
+    MKV_ERR_CUDA = 6,         /* a CUDA runtime call failed (no device, launch error) */
+    MKV_ERR_TIMEOUT = 7,      /* device: a bounded wait inside a kernel ran out       */
+    MKV_ERR_DEVICE_CHECK = 8  /* device: an internal consistency check failed         */
+} mkv_status;
+
+typedef enum { MKV_BF16 = 0, MKV_F32 = 1 } mkv_dtype;
+
+/* Which heads Eq. 4 (Sec. 4.2, "Momentum-Based Attention Aggregation") averages. */
+typedef enum {
+    MKV_SCORE_GROUP_MEAN = 0, /* per KV head: mean over its G query heads; each KV head
+                                 scores and evicts on its own                           */
+    MKV_SCORE_LAYER_MEAN = 1  /* as printed: mean over all H heads, one score vector per
+                                 (layer, sequence), all KV heads evict the same tokens  */
+} mkv_score_mode;
+
+/* Kernel family used for the attention pass. */
+typedef enum {
+    MKV_KERNEL_AUTO = 0, /* tensor-core path where it exists, else the scalar path      */
+    MKV_KERNEL_SIMT = 1, /* scalar fp32 FMA path: every dtype / head_dim                */
+    MKV_KERNEL_MMA = 2   /* bf16, head_dim 128, G <= 8: bulk-copy pipeline + mma        */
+} mkv_kernel;
+
+/* flags for mkv_create */
+#define MKV_FLAG_RECORD_PROBS 1u /* keep the head-averaged decode probabilities of the last
+                                    step (Eq. 4) for mkv_get_last_probs()               */
+
+/*
+ * Size in bytes of the workspace mkv_create() needs for these parameters
+ * (0 if the parameters are invalid).  Pure host arithmetic.  Per cached token and
+ * layer it accounts 2 * kv_heads * head_dim * sizeof(element) bytes (K and V), the
+ * figure Sec. 1 of the paper quotes as 128 KB per token for Llama-3.1-8B at 16 bit.
+ */
+size_t mkv_workspace_bytes(int layers, int batch, int q_heads, int kv_heads, int head_dim,
+                           int budget, int max_prefill, int kv_dtype, int score_mode);
+
+/* K+V bytes one cached token occupies over all layers (the paper's 128 KB/token). */
+size_t mkv_kv_bytes_per_token(int layers, int kv_heads, int head_dim, int kv_dtype);
+
+/*
+ * Create a context (Algorithm 1 "Require": decoding budget B_d = `budget`, momentum
+ * factor alpha = `beta`).
+ *   layers, batch            >= 1
+ *   q_heads % kv_heads == 0; G = q_heads / kv_heads <= 16
+ *   head_dim                 64 or 128
+ *   budget                   >= 1; also the largest budget mkv_set_budget accepts
+ *   beta                     in [0, 1]  (paper: (0,1); 0 and 1 are the limits)
+ *   max_prefill              >= 0, longest prompt any sequence may have
+ *   kv_dtype                 element type of the cache and of q, k_new, v_new
+ *   out_dtype                element type of `out` (MKV_F32 allowed with a bf16 cache)
+ *   score_mode, kernel, flags  see the enums above
+ *   workspace                device pointer, 256-byte aligned, >= mkv_workspace_bytes();
+ *                            its first use zero-fills it on `device`'s legacy stream
+ *   device                   CUDA device ordinal
+ *   out_ctx                  host pointer receiving the context
+ * Errors: INVALID_ARG, UNSUPPORTED (kernel family cannot do this shape), WORKSPACE, CUDA.
+ */
+mkv_status mkv_create(int layers, int q_heads, int kv_heads, int head_dim, int budget, float beta,
+                      int batch, int max_prefill, int kv_dtype, int out_dtype, int score_mode,
+                      int kernel, unsigned flags, void* workspace, size_t workspace_bytes,
+                      int device, mkv_ctx** out_ctx);
+
+/* Frees host state.  The workspace stays with the caller.  NULL is ignored. */
+void mkv_destroy(mkv_ctx* ctx);
+
+/*
+ * Prefill phase (Sec. 4.1): store the prompt's K_P, V_P of one layer in the frozen
+ * prefill pool and empty that layer's decode pool (scores, positions, step counter).
+ *   K, V          device pointers, [batch][kv_heads][src_rows][head_dim], kv_dtype
+ *   prefill_lens  host pointer, [batch]; sequence b uses rows [0, prefill_lens[b])
+ *   src_rows      row count of the source arrays' third index (>= every length)
+ * Asynchronous on `stream`.  Errors: INVALID_ARG, CAPACITY (a length > max_prefill), CUDA.
+ */
+mkv_status mkv_prefill(mkv_ctx* ctx, int layer, const void* K, const void* V,
+                       const int32_t* prefill_lens, int src_rows, void* stream);
+
+/*
+ * One decode step of Algorithm 1 for one layer, all sequences:
+ *   append (k_new, v_new) with importance 0; attention of q over prefill U decode pool
+ *   (Eq. 2), fresh token included; per decode token the head-averaged probability
+ *   (Eq. 4); I <- beta * I + abar (Eq. 5); if the pool holds more than `budget` tokens,
+ *   remove the overflow-many lowest-I tokens (Eq. 7-9; ties: smaller position id first)
+ *   and close the holes.  `out` is the attention output over the pool BEFORE eviction.
+ *   q, k_new, v_new   device pointers, kv_dtype;  out  device pointer, out_dtype
+ * Asynchronous, no allocation, no host synchronisation.
+ * Errors: INVALID_ARG, BAD_STATE (layer not prefilled), CUDA.
+ */
+mkv_status mkv_decode_step(mkv_ctx* ctx, int layer, const void* q, const void* k_new,
+                           const void* v_new, void* out, void* stream);
+
+/*
+ * Same step with HOST buffers: copies q, k_new, v_new to the device, runs the step,
+ * copies `out` back; all on `stream`, asynchronous when the host buffers are pinned
+ * (the caller synchronises the stream before reading `out` or reusing the inputs).
+ */
+mkv_status mkv_decode_step_host(mkv_ctx* ctx, int layer, const void* q_host, const void* k_new_host,
+                                const void* v_new_host, void* out_host, void* stream);
+
+/*
+ * Plain decode attention (Eq. 2) of q over the pools as they are: no append, no score
+ * update, no eviction.  The timing baseline the score/evict overhead is measured against.
+ */
+mkv_status mkv_attend_only(mkv_ctx* ctx, int layer, const void* q, void* out, void* stream);
+
+/*
+ * Change the decode budget B_d (1 <= budget <= the value given to mkv_create).  A
+ * smaller budget makes the next step evict overflow = count - budget > 1 tokens (the
+ * general arg-min of Eq. 8).
+ */
+mkv_status mkv_set_budget(mkv_ctx* ctx, int budget);
+
+/* Back to "no layer prefilled"; pools keep their bytes but are treated as empty. */
+mkv_status mkv_reset(mkv_ctx* ctx);
+
+/* Synchronise `stream`, then return the sticky device status (MKV_OK if clean). */
+mkv_status mkv_status_sync(mkv_ctx* ctx, void* stream);
+
+/* Number of kernels this context has launched so far (host counter). */
+int64_t mkv_launch_count(const mkv_ctx* ctx);
+
+/* ---- inspection: synchronous (device-wide sync + D2H), for tests and debugging ---- */
+
+/* Decode pool of (layer, b, kv_head): *n tokens; pos/score (host, `cap` entries) may be
+ * NULL.  Order is the physical slot order, which compaction permutes. */
+mkv_status mkv_get_decode_state(mkv_ctx* ctx, int layer, int b, int kv_head, int32_t* n,
+                                int32_t* pos, float* score, int cap);
+/* Tokens the last step evicted from that pool, with their scores at eviction. */
+mkv_status mkv_get_last_evicted(mkv_ctx* ctx, int layer, int b, int kv_head, int32_t* k,
+                                int32_t* pos, float* score, int cap);
+/* Eq. 4 values of the last step per slot, pre-eviction order (needs MKV_FLAG_RECORD_PROBS);
+ * *n receives the pre-eviction token count. */
+mkv_status mkv_get_last_probs(mkv_ctx* ctx, int layer, int b, int kv_head, int32_t* n,
+                              float* abar, int cap);
+/* Copy a pool's rows out in plain [token][head_dim] layout (kv_dtype).  pool 0 = prefill,
+ * 1 = decode.  *n receives the token count; at most cap_tokens rows are written. */
+mkv_status mkv_read_kv(mkv_ctx* ctx, int layer, int b, int kv_head, int pool, int32_t* n,
+                       void* K_host, void* V_host, int cap_tokens);
+/* Decode steps completed on a layer since its prefill. */
+mkv_status mkv_get_step(mkv_ctx* ctx, int layer, int64_t* step);
+
+const char* mkv_status_string(mkv_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MKV_H_ */
