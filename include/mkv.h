@@ -37,6 +37,9 @@
 #ifdef __cplusplus
 extern "C" {
 #endif
+#if defined(__GNUC__)
+#pragma GCC visibility push(default) /* the only exported symbols of libmkv.so */
+#endif
 
 typedef struct mkv_ctx mkv_ctx; /* opaque, host-owned */
 
@@ -188,6 +191,9 @@ mkv_status mkv_get_step(mkv_ctx* ctx, int layer, int64_t* step);
 
 const char* mkv_status_string(mkv_status s);
 
+#if defined(__GNUC__)
+#pragma GCC visibility pop
+#endif
 #ifdef __cplusplus
 }
 #endif

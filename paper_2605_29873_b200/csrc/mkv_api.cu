@@ -1,0 +1,525 @@
+// C ABI of the Moment-KV decode library: argument checks, workspace carving, the static
+// work list, launches.  All device work is in the kernels; nothing here computes any
+// step of the method on the host.
+#include <algorithm>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/mkv.h"
+#include "mkv_launch.h"
+
+using namespace mkv;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline int round16(int a) { return (a + 15) / 16 * 16; }
+inline int elem_size(int dt) { return dt == MKV_BF16 ? 2 : 4; }
+
+// smallest item size the work list may ever use for this shape: bounds the number of
+// partials per unit (kMaxParts) and therefore the scratch the workspace must hold
+int min_item_rows(int max_prefill, int cap) {
+    const int need = round16(ceil_div(max_prefill + cap, kMaxParts - 2));
+    return std::max(64, need);
+}
+
+struct LayerOff {
+    size_t Kp, Vp, Kd, Vd, score, pos, n_dec, logit, abar, n_prev, ev_k, ev_pos, ev_score, items, unit_lp,
+        unit_part0, unit_nparts, part_o, part_ml, ticket, sched, step, keys, list_a, list_b, end;
+};
+struct Layout {
+    int units, cap, rowb, max_items;
+    size_t status, stage_q, stage_k, stage_v, stage_out, layer0, layer_bytes, total;
+    LayerOff lo;  // offsets relative to the layer base
+};
+
+bool make_layout(int layers, int batch, int q_heads, int kv_heads, int head_dim, int budget, int max_prefill,
+                 int kv_dtype, Layout* out) {
+    if (layers < 1 || batch < 1 || q_heads < 1 || kv_heads < 1 || budget < 1 || max_prefill < 0) return false;
+    if (q_heads % kv_heads) return false;
+    if (head_dim != 64 && head_dim != 128) return false;
+    if (kv_dtype != MKV_BF16 && kv_dtype != MKV_F32) return false;
+    const int G = q_heads / kv_heads;
+    if (G > kMaxGroup) return false;
+    if ((long long)budget + 1 > (1 << 24) || max_prefill > (1 << 24)) return false;
+    Layout L;
+    L.units = batch * kv_heads;
+    L.cap = budget + 1;
+    L.rowb = head_dim * elem_size(kv_dtype);
+    const int irm = min_item_rows(max_prefill, L.cap);
+    L.max_items = L.units * (ceil_div(max_prefill, irm) + ceil_div(L.cap, irm));
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes); return r; };
+    L.status = take(256);
+    L.stage_q = take((size_t)batch * q_heads * head_dim * 4);
+    L.stage_k = take((size_t)batch * kv_heads * head_dim * 4);
+    L.stage_v = take((size_t)batch * kv_heads * head_dim * 4);
+    L.stage_out = take((size_t)batch * q_heads * head_dim * 4);
+    L.layer0 = o;
+    o = 0;
+    const size_t U = (size_t)L.units, C = (size_t)L.cap;
+    L.lo.Kp = take(U * max_prefill * L.rowb);
+    L.lo.Vp = take(U * max_prefill * L.rowb);
+    L.lo.Kd = take(U * C * L.rowb);
+    L.lo.Vd = take(U * C * L.rowb);
+    L.lo.score = take(U * C * 4);
+    L.lo.pos = take(U * C * 4);
+    L.lo.n_dec = take(U * 4);
+    L.lo.logit = take((size_t)batch * q_heads * C * 4);
+    L.lo.abar = take(U * C * 4);
+    L.lo.n_prev = take(U * 4);
+    L.lo.ev_k = take(U * 4);
+    L.lo.ev_pos = take(U * C * 4);
+    L.lo.ev_score = take(U * C * 4);
+    L.lo.items = take((size_t)L.max_items * sizeof(Item));
+    L.lo.unit_lp = take(U * 4);
+    L.lo.unit_part0 = take(U * 4);
+    L.lo.unit_nparts = take(U * 4);
+    L.lo.part_o = take((size_t)L.max_items * G * head_dim * 4);
+    L.lo.part_ml = take((size_t)L.max_items * G * 2 * 4);
+    L.lo.ticket = take(U * 4);
+    L.lo.sched = take(256);
+    L.lo.step = take(256);
+    L.lo.keys = take(U * C * 8);
+    L.lo.list_a = take(U * C * 4);
+    L.lo.list_b = take(U * C * 4);
+    L.lo.end = o;
+    L.layer_bytes = o;
+    L.total = L.layer0 + L.layer_bytes * (size_t)layers;
+    *out = L;
+    return true;
+}
+
+// Copies source rows [units][src_rows][rowb] into the chunk-permuted pool rows.
+__global__ void prefill_copy_kernel(const uint8_t* __restrict__ srcK, const uint8_t* __restrict__ srcV,
+                                    uint8_t* __restrict__ dstK, uint8_t* __restrict__ dstV,
+                                    const int32_t* __restrict__ unit_lp, int units, int src_rows, int max_prefill,
+                                    int rowb) {
+    const int chunks = rowb >> 4;
+    const long long per_unit = (long long)src_rows * chunks;
+    const long long total = per_unit * units;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        const int u = (int)(i / per_unit);
+        const long long r = i - (long long)u * per_unit;
+        const int row = (int)(r / chunks), c = (int)(r - (long long)row * chunks);
+        if (row >= unit_lp[u]) continue;
+        const size_t s = ((size_t)u * src_rows + row) * rowb + (size_t)c * 16;
+        const size_t d = ((size_t)u * max_prefill + row) * rowb + (size_t)((c ^ (row & 7)) * 16);
+        *reinterpret_cast<uint4*>(dstK + d) = *reinterpret_cast<const uint4*>(srcK + s);
+        *reinterpret_cast<uint4*>(dstV + d) = *reinterpret_cast<const uint4*>(srcV + s);
+    }
+}
+
+}  // namespace
+
+struct mkv_ctx {
+    int layers, batch, q_heads, kv_heads, head_dim, group;
+    int budget, budget_max, max_prefill;
+    float beta;
+    int kv_dtype, out_dtype, score_mode, kernel;
+    unsigned flags;
+    int device;
+    uint8_t* ws;
+    Layout lay;
+    int item_rows;
+    int n_ctas;     // persistent grid of the tensor-core kernel
+    bool use_mma;
+    std::vector<char> prefilled;
+    std::vector<int> n_items;
+    std::vector<std::vector<int32_t>> lens;   // per layer, per sequence
+    int64_t launches;
+};
+
+namespace {
+
+LayerDev layer_dev(const mkv_ctx* c, int layer) {
+    uint8_t* base = c->ws + c->lay.layer0 + c->lay.layer_bytes * (size_t)layer;
+    const LayerOff& o = c->lay.lo;
+    LayerDev d;
+    d.Kp = base + o.Kp; d.Vp = base + o.Vp; d.Kd = base + o.Kd; d.Vd = base + o.Vd;
+    d.score = (float*)(base + o.score);
+    d.pos = (int32_t*)(base + o.pos);
+    d.n_dec = (int32_t*)(base + o.n_dec);
+    d.logit = (float*)(base + o.logit);
+    d.abar = (c->flags & MKV_FLAG_RECORD_PROBS) ? (float*)(base + o.abar) : nullptr;
+    d.n_prev = (int32_t*)(base + o.n_prev);
+    d.ev_k = (int32_t*)(base + o.ev_k);
+    d.ev_pos = (int32_t*)(base + o.ev_pos);
+    d.ev_score = (float*)(base + o.ev_score);
+    d.items = (const Item*)(base + o.items);
+    d.n_items = c->n_items[layer];
+    d.unit_lp = (const int32_t*)(base + o.unit_lp);
+    d.unit_part0 = (const int32_t*)(base + o.unit_part0);
+    d.unit_nparts = (const int32_t*)(base + o.unit_nparts);
+    d.part_o = (float*)(base + o.part_o);
+    d.part_ml = (float*)(base + o.part_ml);
+    d.ticket = (int32_t*)(base + o.ticket);
+    d.sched = (int32_t*)(base + o.sched);
+    d.step = (int32_t*)(base + o.step);
+    d.keys = (unsigned long long*)(base + o.keys);
+    d.list_a = (int32_t*)(base + o.list_a);
+    d.list_b = (int32_t*)(base + o.list_b);
+    return d;
+}
+
+Params make_params(const mkv_ctx* c, int layer, const void* q, const void* k_new, const void* v_new, void* out,
+                   int mode) {
+    Params p;
+    p.L = layer_dev(c, layer);
+    p.q = q; p.k_new = k_new; p.v_new = v_new; p.out = out;
+    p.status = (int32_t*)(c->ws + c->lay.status);
+    p.batch = c->batch; p.q_heads = c->q_heads; p.kv_heads = c->kv_heads; p.group = c->group;
+    p.head_dim = c->head_dim;
+    p.cap = c->lay.cap; p.max_prefill = c->max_prefill; p.budget = c->budget;
+    p.beta = c->beta;
+    p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c->head_dim));
+    p.mode = mode;
+    p.out_f32 = (c->out_dtype == MKV_F32);
+    return p;
+}
+
+mkv_status launch_step(mkv_ctx* c, const Params& p, cudaStream_t st) {
+    cudaError_t e = c->use_mma ? launch_mma(p, c->n_ctas, st) : launch_simt(p, c->kv_dtype, st);
+    if (e != cudaSuccess) return MKV_ERR_CUDA;
+    c->launches += 1;
+    return MKV_OK;
+}
+
+bool layer_ok(const mkv_ctx* c, int layer) { return c && layer >= 0 && layer < c->layers; }
+
+struct DeviceGuard {
+    int prev = -1; bool ok;
+    explicit DeviceGuard(int dev) {
+        ok = cudaGetDevice(&prev) == cudaSuccess;
+        if (ok && prev != dev) ok = cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+}  // namespace
+
+extern "C" {
+
+size_t mkv_workspace_bytes(int layers, int batch, int q_heads, int kv_heads, int head_dim, int budget,
+                           int max_prefill, int kv_dtype, int score_mode) {
+    (void)score_mode;
+    Layout L;
+    if (!make_layout(layers, batch, q_heads, kv_heads, head_dim, budget, max_prefill, kv_dtype, &L)) return 0;
+    return L.total;
+}
+
+size_t mkv_kv_bytes_per_token(int layers, int kv_heads, int head_dim, int kv_dtype) {
+    if (layers < 1 || kv_heads < 1 || head_dim < 1 || (kv_dtype != MKV_BF16 && kv_dtype != MKV_F32)) return 0;
+    return (size_t)layers * kv_heads * 2 * head_dim * elem_size(kv_dtype);
+}
+
+mkv_status mkv_create(int layers, int q_heads, int kv_heads, int head_dim, int budget, float beta, int batch,
+                      int max_prefill, int kv_dtype, int out_dtype, int score_mode, int kernel, unsigned flags,
+                      void* workspace, size_t workspace_bytes, int device, mkv_ctx** out_ctx) {
+    if (!out_ctx) return MKV_ERR_INVALID_ARG;
+    *out_ctx = nullptr;
+    Layout L;
+    if (!make_layout(layers, batch, q_heads, kv_heads, head_dim, budget, max_prefill, kv_dtype, &L))
+        return MKV_ERR_INVALID_ARG;
+    if (!(beta >= 0.0f && beta <= 1.0f)) return MKV_ERR_INVALID_ARG;
+    if (out_dtype != MKV_BF16 && out_dtype != MKV_F32) return MKV_ERR_INVALID_ARG;
+    if (kv_dtype == MKV_F32 && out_dtype != MKV_F32) return MKV_ERR_INVALID_ARG;
+    if (score_mode != MKV_SCORE_GROUP_MEAN && score_mode != MKV_SCORE_LAYER_MEAN) return MKV_ERR_INVALID_ARG;
+    if (kernel < MKV_KERNEL_AUTO || kernel > MKV_KERNEL_MMA) return MKV_ERR_INVALID_ARG;
+    if (flags & ~MKV_FLAG_RECORD_PROBS) return MKV_ERR_INVALID_ARG;
+    if (!workspace || device < 0) return MKV_ERR_INVALID_ARG;
+    const int G = q_heads / kv_heads;
+    if (score_mode == MKV_SCORE_LAYER_MEAN && kv_heads != 1) return MKV_ERR_UNSUPPORTED;
+    const bool mma_ok = mma_supported(kv_dtype, head_dim, G);
+    const bool simt_ok = simt_supported(kv_dtype, head_dim, G);
+    bool use_mma;
+    if (kernel == MKV_KERNEL_MMA) { if (!mma_ok) return MKV_ERR_UNSUPPORTED; use_mma = true; }
+    else if (kernel == MKV_KERNEL_SIMT) { if (!simt_ok) return MKV_ERR_UNSUPPORTED; use_mma = false; }
+    else { if (!mma_ok && !simt_ok) return MKV_ERR_UNSUPPORTED; use_mma = mma_ok; }
+    if (((uintptr_t)workspace % kAlign) != 0 || workspace_bytes < L.total) return MKV_ERR_WORKSPACE;
+
+    DeviceGuard guard(device);
+    if (!guard.ok) return MKV_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return MKV_ERR_CUDA;
+    if (use_mma && mma_configure() != cudaSuccess) return MKV_ERR_CUDA;
+    // Zero everything once: counters, tickets, status, and the pools (rows that are never
+    // written must still hold finite numbers because masked rows enter 0 * v products).
+    if (cudaMemset(workspace, 0, L.total) != cudaSuccess) return MKV_ERR_CUDA;
+    if (cudaDeviceSynchronize() != cudaSuccess) return MKV_ERR_CUDA;
+
+    mkv_ctx* c = new (std::nothrow) mkv_ctx();
+    if (!c) return MKV_ERR_INVALID_ARG;
+    c->layers = layers; c->batch = batch; c->q_heads = q_heads; c->kv_heads = kv_heads;
+    c->head_dim = head_dim; c->group = G;
+    c->budget = budget; c->budget_max = budget; c->max_prefill = max_prefill; c->beta = beta;
+    c->kv_dtype = kv_dtype; c->out_dtype = out_dtype; c->score_mode = score_mode; c->kernel = kernel;
+    c->flags = flags; c->device = device; c->ws = (uint8_t*)workspace; c->lay = L;
+    c->use_mma = use_mma;
+    int ir = 256;
+    if (const char* e = std::getenv("MKV_ITEM_ROWS")) ir = std::atoi(e);
+    c->item_rows = std::max(min_item_rows(max_prefill, L.cap), round16(std::max(ir, 16)));
+    int per_sm = 2;
+    if (const char* e = std::getenv("MKV_CTAS_PER_SM")) per_sm = std::max(1, std::min(4, std::atoi(e)));
+    c->n_ctas = prop.multiProcessorCount * per_sm;
+    c->prefilled.assign(layers, 0);
+    c->n_items.assign(layers, 0);
+    c->lens.assign(layers, std::vector<int32_t>(batch, 0));
+    c->launches = 0;
+    *out_ctx = c;
+    return MKV_OK;
+}
+
+void mkv_destroy(mkv_ctx* ctx) { delete ctx; }
+
+mkv_status mkv_prefill(mkv_ctx* c, int layer, const void* K, const void* V, const int32_t* prefill_lens,
+                       int src_rows, void* stream) {
+    if (!layer_ok(c, layer) || !prefill_lens || src_rows < 0) return MKV_ERR_INVALID_ARG;
+    int maxlen = 0;
+    for (int b = 0; b < c->batch; ++b) {
+        if (prefill_lens[b] < 0 || prefill_lens[b] > src_rows) return MKV_ERR_INVALID_ARG;
+        if (prefill_lens[b] > c->max_prefill) return MKV_ERR_CAPACITY;
+        maxlen = std::max(maxlen, prefill_lens[b]);
+    }
+    if (maxlen > 0 && (!K || !V)) return MKV_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MKV_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    const Layout& L = c->lay;
+    const int U = L.units, cap = L.cap, ir = c->item_rows;
+
+    // static work list: unit-major, prefill segment then decode segment, pieces of equal
+    // size (a multiple of 16 rows) no longer than item_rows
+    std::vector<Item> items;
+    std::vector<int32_t> lp(U), part0(U), nparts(U);
+    for (int u = 0; u < U; ++u) {
+        const int len = prefill_lens[u / c->kv_heads];
+        lp[u] = len;
+        part0[u] = (int32_t)items.size();
+        for (int seg = 0; seg < 2; ++seg) {
+            const int total = seg == 0 ? len : cap;
+            if (total == 0) continue;
+            const int pieces = ceil_div(total, ir);
+            const int piece = round16(ceil_div(total, pieces));
+            for (int r0 = 0; r0 < total; r0 += piece) items.push_back(Item{u, r0, std::min(piece, total - r0), seg});
+        }
+        nparts[u] = (int32_t)items.size() - part0[u];
+        if (nparts[u] > kMaxParts) return MKV_ERR_CAPACITY;
+    }
+    if ((int)items.size() > L.max_items) return MKV_ERR_CAPACITY;
+    c->n_items[layer] = (int)items.size();
+    for (int b = 0; b < c->batch; ++b) c->lens[layer][b] = prefill_lens[b];
+
+    uint8_t* base = c->ws + L.layer0 + L.layer_bytes * (size_t)layer;
+    bool ok = true;
+    ok &= cudaMemcpyAsync(base + L.lo.items, items.data(), items.size() * sizeof(Item), cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(base + L.lo.unit_lp, lp.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(base + L.lo.unit_part0, part0.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(base + L.lo.unit_nparts, nparts.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    // empty decode pool, rewind counters
+    ok &= cudaMemsetAsync(base + L.lo.n_dec, 0, U * 4, st) == cudaSuccess;
+    ok &= cudaMemsetAsync(base + L.lo.n_prev, 0, U * 4, st) == cudaSuccess;
+    ok &= cudaMemsetAsync(base + L.lo.ev_k, 0, U * 4, st) == cudaSuccess;
+    ok &= cudaMemsetAsync(base + L.lo.ticket, 0, U * 4, st) == cudaSuccess;
+    ok &= cudaMemsetAsync(base + L.lo.sched, 0, 256, st) == cudaSuccess;
+    ok &= cudaMemsetAsync(base + L.lo.step, 0, 256, st) == cudaSuccess;
+    if (!ok) return MKV_ERR_CUDA;
+    // host vectors above are pageable: the runtime has staged them before returning
+    if (maxlen > 0) {
+        const long long total = (long long)U * src_rows * (L.rowb / 16);
+        const int threads = 256;
+        const int blocks = (int)std::min<long long>((total + threads - 1) / threads, 148 * 16);
+        prefill_copy_kernel<<<blocks, threads, 0, st>>>((const uint8_t*)K, (const uint8_t*)V, base + L.lo.Kp,
+                                                        base + L.lo.Vp, (const int32_t*)(base + L.lo.unit_lp), U,
+                                                        src_rows, c->max_prefill, L.rowb);
+        if (cudaGetLastError() != cudaSuccess) return MKV_ERR_CUDA;
+        c->launches += 1;
+    }
+    c->prefilled[layer] = 1;
+    return MKV_OK;
+}
+
+mkv_status mkv_decode_step(mkv_ctx* c, int layer, const void* q, const void* k_new, const void* v_new, void* out,
+                           void* stream) {
+    if (!layer_ok(c, layer) || !q || !k_new || !v_new || !out) return MKV_ERR_INVALID_ARG;
+    if (!c->prefilled[layer]) return MKV_ERR_BAD_STATE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MKV_ERR_CUDA;
+    const Params p = make_params(c, layer, q, k_new, v_new, out, kModeDecode);
+    return launch_step(c, p, (cudaStream_t)stream);
+}
+
+mkv_status mkv_decode_step_host(mkv_ctx* c, int layer, const void* qh, const void* kh, const void* vh, void* outh,
+                                void* stream) {
+    if (!layer_ok(c, layer) || !qh || !kh || !vh || !outh) return MKV_ERR_INVALID_ARG;
+    if (!c->prefilled[layer]) return MKV_ERR_BAD_STATE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MKV_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t es = elem_size(c->kv_dtype), os = elem_size(c->out_dtype);
+    const size_t nq = (size_t)c->batch * c->q_heads * c->head_dim, nk = (size_t)c->batch * c->kv_heads * c->head_dim;
+    uint8_t *dq = c->ws + c->lay.stage_q, *dk = c->ws + c->lay.stage_k, *dv = c->ws + c->lay.stage_v,
+            *dout = c->ws + c->lay.stage_out;
+    if (cudaMemcpyAsync(dq, qh, nq * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return MKV_ERR_CUDA;
+    if (cudaMemcpyAsync(dk, kh, nk * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return MKV_ERR_CUDA;
+    if (cudaMemcpyAsync(dv, vh, nk * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return MKV_ERR_CUDA;
+    const Params p = make_params(c, layer, dq, dk, dv, dout, kModeDecode);
+    const mkv_status s = launch_step(c, p, st);
+    if (s != MKV_OK) return s;
+    if (cudaMemcpyAsync(outh, dout, nq * os, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MKV_ERR_CUDA;
+    return MKV_OK;
+}
+
+mkv_status mkv_attend_only(mkv_ctx* c, int layer, const void* q, void* out, void* stream) {
+    if (!layer_ok(c, layer) || !q || !out) return MKV_ERR_INVALID_ARG;
+    if (!c->prefilled[layer]) return MKV_ERR_BAD_STATE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MKV_ERR_CUDA;
+    const Params p = make_params(c, layer, q, nullptr, nullptr, out, kModeAttendOnly);
+    return launch_step(c, p, (cudaStream_t)stream);
+}
+
+mkv_status mkv_set_budget(mkv_ctx* c, int budget) {
+    if (!c || budget < 1) return MKV_ERR_INVALID_ARG;
+    if (budget > c->budget_max) return MKV_ERR_CAPACITY;
+    c->budget = budget;
+    return MKV_OK;
+}
+
+mkv_status mkv_reset(mkv_ctx* c) {
+    if (!c) return MKV_ERR_INVALID_ARG;
+    std::fill(c->prefilled.begin(), c->prefilled.end(), 0);
+    c->budget = c->budget_max;
+    return MKV_OK;
+}
+
+mkv_status mkv_status_sync(mkv_ctx* c, void* stream) {
+    if (!c) return MKV_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MKV_ERR_CUDA;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return MKV_ERR_CUDA;
+    int32_t s = 0;
+    if (cudaMemcpy(&s, c->ws + c->lay.status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return MKV_ERR_CUDA;
+    return (mkv_status)s;
+}
+
+int64_t mkv_launch_count(const mkv_ctx* c) { return c ? c->launches : 0; }
+
+static mkv_status unit_args(mkv_ctx* c, int layer, int b, int g) {
+    if (!layer_ok(c, layer) || b < 0 || b >= c->batch || g < 0 || g >= c->kv_heads) return MKV_ERR_INVALID_ARG;
+    if (!c->prefilled[layer]) return MKV_ERR_BAD_STATE;
+    return MKV_OK;
+}
+#define MKV_D2H(dst, src, bytes) \
+    do { if ((bytes) > 0 && cudaMemcpy((dst), (src), (bytes), cudaMemcpyDeviceToHost) != cudaSuccess) return MKV_ERR_CUDA; } while (0)
+
+mkv_status mkv_get_decode_state(mkv_ctx* c, int layer, int b, int g, int32_t* n, int32_t* pos, float* score,
+                                int cap) {
+    mkv_status s = unit_args(c, layer, b, g);
+    if (s != MKV_OK) return s;
+    if (!n) return MKV_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok || cudaDeviceSynchronize() != cudaSuccess) return MKV_ERR_CUDA;
+    const LayerDev d = layer_dev(c, layer);
+    const int u = b * c->kv_heads + g;
+    MKV_D2H(n, d.n_dec + u, 4);
+    if ((pos || score) && *n > cap) return MKV_ERR_CAPACITY;
+    if (pos) MKV_D2H(pos, d.pos + (size_t)u * c->lay.cap, (size_t)*n * 4);
+    if (score) MKV_D2H(score, d.score + (size_t)u * c->lay.cap, (size_t)*n * 4);
+    return MKV_OK;
+}
+
+mkv_status mkv_get_last_evicted(mkv_ctx* c, int layer, int b, int g, int32_t* k, int32_t* pos, float* score,
+                                int cap) {
+    mkv_status s = unit_args(c, layer, b, g);
+    if (s != MKV_OK) return s;
+    if (!k) return MKV_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok || cudaDeviceSynchronize() != cudaSuccess) return MKV_ERR_CUDA;
+    const LayerDev d = layer_dev(c, layer);
+    const int u = b * c->kv_heads + g;
+    MKV_D2H(k, d.ev_k + u, 4);
+    if ((pos || score) && *k > cap) return MKV_ERR_CAPACITY;
+    if (pos) MKV_D2H(pos, d.ev_pos + (size_t)u * c->lay.cap, (size_t)*k * 4);
+    if (score) MKV_D2H(score, d.ev_score + (size_t)u * c->lay.cap, (size_t)*k * 4);
+    return MKV_OK;
+}
+
+mkv_status mkv_get_last_probs(mkv_ctx* c, int layer, int b, int g, int32_t* n, float* abar, int cap) {
+    mkv_status s = unit_args(c, layer, b, g);
+    if (s != MKV_OK) return s;
+    if (!n) return MKV_ERR_INVALID_ARG;
+    if (!(c->flags & MKV_FLAG_RECORD_PROBS)) return MKV_ERR_BAD_STATE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok || cudaDeviceSynchronize() != cudaSuccess) return MKV_ERR_CUDA;
+    const LayerDev d = layer_dev(c, layer);
+    const int u = b * c->kv_heads + g;
+    MKV_D2H(n, d.n_prev + u, 4);
+    if (abar && *n > cap) return MKV_ERR_CAPACITY;
+    if (abar) MKV_D2H(abar, d.abar + (size_t)u * c->lay.cap, (size_t)*n * 4);
+    return MKV_OK;
+}
+
+mkv_status mkv_read_kv(mkv_ctx* c, int layer, int b, int g, int pool, int32_t* n, void* Kh, void* Vh,
+                       int cap_tokens) {
+    mkv_status s = unit_args(c, layer, b, g);
+    if (s != MKV_OK) return s;
+    if (!n || (pool != 0 && pool != 1) || cap_tokens < 0) return MKV_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok || cudaDeviceSynchronize() != cudaSuccess) return MKV_ERR_CUDA;
+    const LayerDev d = layer_dev(c, layer);
+    const int u = b * c->kv_heads + g;
+    const int rowb = c->lay.rowb;
+    int count;
+    size_t base;
+    if (pool == 0) { count = c->lens[layer][b]; base = (size_t)u * c->max_prefill * rowb; }
+    else { MKV_D2H(&count, d.n_dec + u, 4); base = (size_t)u * c->lay.cap * rowb; }
+    *n = count;
+    const int rows = std::min(count, cap_tokens);
+    if (rows == 0 || (!Kh && !Vh)) return MKV_OK;
+    std::vector<uint8_t> raw((size_t)rows * rowb);
+    for (int which = 0; which < 2; ++which) {
+        uint8_t* dst = (uint8_t*)(which == 0 ? Kh : Vh);
+        if (!dst) continue;
+        const uint8_t* src = (pool == 0 ? (which == 0 ? d.Kp : d.Vp) : (which == 0 ? d.Kd : d.Vd)) + base;
+        MKV_D2H(raw.data(), src, raw.size());
+        for (int r = 0; r < rows; ++r)
+            for (int ch = 0; ch < rowb / 16; ++ch)
+                std::memcpy(dst + (size_t)r * rowb + ch * 16, raw.data() + (size_t)r * rowb + ((ch ^ (r & 7)) * 16), 16);
+    }
+    return MKV_OK;
+}
+
+mkv_status mkv_get_step(mkv_ctx* c, int layer, int64_t* step) {
+    if (!layer_ok(c, layer) || !step) return MKV_ERR_INVALID_ARG;
+    if (!c->prefilled[layer]) return MKV_ERR_BAD_STATE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok || cudaDeviceSynchronize() != cudaSuccess) return MKV_ERR_CUDA;
+    int32_t s = 0;
+    MKV_D2H(&s, layer_dev(c, layer).step, 4);
+    *step = s;
+    return MKV_OK;
+}
+
+const char* mkv_status_string(mkv_status s) {
+    switch (s) {
+        case MKV_OK: return "ok";
+        case MKV_ERR_INVALID_ARG: return "invalid argument";
+        case MKV_ERR_BAD_STATE: return "bad state";
+        case MKV_ERR_CAPACITY: return "capacity exceeded";
+        case MKV_ERR_WORKSPACE: return "workspace too small or misaligned";
+        case MKV_ERR_UNSUPPORTED: return "unsupported configuration";
+        case MKV_ERR_CUDA: return "CUDA runtime error";
+        case MKV_ERR_TIMEOUT: return "device wait timed out";
+        case MKV_ERR_DEVICE_CHECK: return "device consistency check failed";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,14 @@
+// Host-side launch entry points of the kernel families (internal to the library).
+#pragma once
+#include <cuda_runtime.h>
+
+#include "mkv_common.cuh"
+
+namespace mkv {
+// returns false when no instantiation exists for (dtype, head_dim, group)
+bool simt_supported(int kv_dtype, int head_dim, int group);
+cudaError_t launch_simt(const Params& p, int kv_dtype, cudaStream_t stream);
+bool mma_supported(int kv_dtype, int head_dim, int group);
+cudaError_t launch_mma(const Params& p, int n_ctas, cudaStream_t stream);
+cudaError_t mma_configure();   // one-time function attributes (dynamic shared memory)
+}  // namespace mkv

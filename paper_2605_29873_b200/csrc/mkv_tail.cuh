@@ -1,0 +1,220 @@
+// Tail of one unit (sequence b, KV head g), run by the thread group that delivered the
+// unit's last partial.  In order:
+//   1. cross-split log-sum-exp combine: global max M_h and sum L_h per query head,
+//      out_h = sum_p O_p 2^(m_p - M_h) / L_h                      (Eq. 2)
+//   2. normalised probability of every decode token, including the fresh one, from the
+//      stored raw logits: p = 2^(s - M_h) / L_h; mean over the G heads  (Eq. 4)
+//   3. I_i <- beta * I_i + abar_i, the fresh token starting from 0    (Eq. 5, Eq. 6)
+//   4. overflow k = max(0, n - budget) (Eq. 7); the k smallest 64-bit keys
+//      (fp32 score bits, position id) are the evicted set (Eq. 8).  Scores are
+//      non-negative so their bit patterns order like the values: selection is integer
+//      work on exactly the scores that are stored.  k = 1: arg-min reduction.
+//      k > 1: 8-pass byte-wise radix select of the k-th key.
+//   5. compaction (Eq. 9): survivors stored beyond the new count move into the holes
+//      (K row, V row, score, position id); slot order changes, which is harmless because
+//      softmax and sum(p v) do not depend on the order and ties are broken by position id.
+// NT threads take part (a multiple of 32); they synchronise on named barrier BAR only,
+// so a subset of a CTA can run the tail while other warps keep streaming.
+#pragma once
+#include "mkv_common.cuh"
+
+namespace mkv {
+
+template <int NT>
+struct TailSmem {
+    float M[kMaxGroup];
+    float invL[kMaxGroup];
+    float w[kMaxParts][kMaxGroup];
+    unsigned long long red_key[NT / 32];
+    int red_slot[NT / 32];
+    int hist[256];
+    int cnt[3][NT / 32];
+    int misc[4];
+};
+
+__device__ inline void copy_row_swizzled(uint8_t* pool, size_t unit_base, int rowb, int src, int dst,
+                                         int lane) {
+    const int chunks = rowb >> 4;
+    const uint4* s = reinterpret_cast<const uint4*>(pool + unit_base + (size_t)src * rowb);
+    uint4* d = reinterpret_cast<uint4*>(pool + unit_base + (size_t)dst * rowb);
+    for (int c = lane; c < chunks; c += 32) d[c ^ (dst & 7)] = __ldcg(&s[c ^ (src & 7)]);
+}
+
+template <int NT, int BAR>
+__device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid, int rowb) {
+    const LayerDev& L = p.L;
+    const int G = p.group, D = p.head_dim, cap = p.cap;
+    const int b = u / p.kv_heads, g = u - b * p.kv_heads;
+    const int P = L.unit_nparts[u], part0 = L.unit_part0[u];
+    const int n_old = L.n_dec[u];
+    const bool dec = (p.mode == kModeDecode);
+    const int n = dec ? min(n_old + 1, cap) : n_old;
+    const int lane = tid & 31, warp = tid >> 5;
+    constexpr int NW = NT / 32;
+
+    // ---- 1. combine -------------------------------------------------------------------
+    if (tid < G) {
+        float M = kNegBig;
+        for (int q = 0; q < P; ++q) M = fmaxf(M, __ldcg(&L.part_ml[((size_t)(part0 + q) * G + tid) * 2]));
+        float Lsum = 0.f;
+        for (int q = 0; q < P; ++q) {
+            const float2 ml = __ldcg(reinterpret_cast<const float2*>(&L.part_ml[((size_t)(part0 + q) * G + tid) * 2]));
+            const float w = fast_exp2(ml.x - M);
+            sm.w[q][tid] = w;
+            Lsum += ml.y * w;
+        }
+        sm.M[tid] = M;
+        sm.invL[tid] = Lsum > 0.f ? 1.0f / Lsum : 0.f;
+    }
+    bar_sync(BAR, NT);
+    {
+        const size_t obase = ((size_t)b * p.q_heads + (size_t)g * G) * D;
+        for (int idx = tid; idx < G * D; idx += NT) {
+            const int h = idx / D;
+            float acc = 0.f;
+            for (int q = 0; q < P; ++q)
+                acc = fmaf(__ldcg(&L.part_o[(size_t)(part0 + q) * G * D + idx]), sm.w[q][h], acc);
+            acc *= sm.invL[h];
+            if (p.out_f32) reinterpret_cast<float*>(p.out)[obase + idx] = acc;
+            else reinterpret_cast<__nv_bfloat16*>(p.out)[obase + idx] = __float2bfloat16_rn(acc);
+        }
+    }
+    if (!dec) {
+        if (tid == 0) L.ticket[u] = 0;
+        return;
+    }
+
+    // ---- 2./3. probabilities, head mean, momentum update ---------------------------------
+    const int t = L.step[0];
+    const int k = max(0, n - p.budget);
+    const float inv_g = 1.0f / (float)G;
+    float* score = L.score + (size_t)u * cap;
+    int32_t* pos = L.pos + (size_t)u * cap;
+    unsigned long long* keys = L.keys + (size_t)u * cap;
+    const float* lg = L.logit + ((size_t)b * p.q_heads + (size_t)g * G) * cap;
+    unsigned long long best_key = ~0ull;
+    int best_slot = -1;
+    for (int i = tid; i < n; i += NT) {
+        float s = 0.f;
+        for (int h = 0; h < G; ++h) s += fast_exp2(__ldcg(&lg[(size_t)h * cap + i]) - sm.M[h]) * sm.invL[h];
+        const float ab = s * inv_g;
+        const bool fresh = (i == n - 1);
+        const float old = fresh ? 0.f : score[i];
+        const float nw = fmaf(p.beta, old, ab);
+        const int ps = fresh ? t : pos[i];
+        score[i] = nw;
+        if (fresh) pos[i] = t;
+        if (L.abar) L.abar[(size_t)u * cap + i] = ab;
+        const unsigned long long key = ((unsigned long long)__float_as_uint(nw) << 32) | (unsigned)ps;
+        if (k > 1) keys[i] = key;
+        if (key < best_key) { best_key = key; best_slot = i; }
+    }
+    if (tid == 0) { L.n_prev[u] = n; L.ev_k[u] = k; L.n_dec[u] = n - k; }
+    if (k == 0) {
+        if (tid == 0) L.ticket[u] = 0;
+        return;
+    }
+
+    const size_t ubase = (size_t)u * cap * rowb;
+    if (k == 1) {
+        // ---- 4a. arg-min over (score bits, position id) ------------------------------
+        for (int off = 16; off; off >>= 1) {
+            const unsigned long long ok = __shfl_xor_sync(0xffffffffu, best_key, off);
+            const int os = __shfl_xor_sync(0xffffffffu, best_slot, off);
+            if (ok < best_key) { best_key = ok; best_slot = os; }
+        }
+        if (lane == 0) { sm.red_key[warp] = best_key; sm.red_slot[warp] = best_slot; }
+        bar_sync(BAR, NT);   // also orders every score/pos write before the move below
+        unsigned long long kk = sm.red_key[0];
+        int e = sm.red_slot[0];
+        for (int w2 = 1; w2 < NW; ++w2)
+            if (sm.red_key[w2] < kk) { kk = sm.red_key[w2]; e = sm.red_slot[w2]; }
+        // ---- 5a. the fresh slot n-1 is the only possible mover ------------------------
+        if (tid == 0) {
+            L.ev_pos[(size_t)u * cap] = (int32_t)(unsigned)(kk & 0xffffffffu);
+            L.ev_score[(size_t)u * cap] = __uint_as_float((unsigned)(kk >> 32));
+        }
+        if (e != n - 1) {
+            if (warp == 0) copy_row_swizzled(L.Kd, ubase, rowb, n - 1, e, lane);
+            if (warp == (NW > 1 ? 1 : 0)) copy_row_swizzled(L.Vd, ubase, rowb, n - 1, e, lane);
+            if (tid == NT - 1) { score[e] = score[n - 1]; pos[e] = pos[n - 1]; }
+        }
+        if (tid == 0) L.ticket[u] = 0;
+        return;
+    }
+
+    // ---- 4b. radix select of the k-th smallest key (keys are distinct) ----------------
+    unsigned long long prefix = 0ull, mask = 0ull;
+    int want = k - 1;
+    for (int pass = 7; pass >= 0; --pass) {
+        for (int i = tid; i < 256; i += NT) sm.hist[i] = 0;
+        bar_sync(BAR, NT);
+        for (int i = tid; i < n; i += NT) {
+            const unsigned long long key = keys[i];
+            if ((key & mask) == prefix) atomicAdd(&sm.hist[(int)((key >> (8 * pass)) & 255ull)], 1);
+        }
+        bar_sync(BAR, NT);
+        if (tid == 0) {
+            int cum = 0, sel = 255;
+            for (int bin = 0; bin < 256; ++bin) {
+                const int c = sm.hist[bin];
+                if (want < cum + c) { sel = bin; break; }
+                cum += c;
+            }
+            sm.misc[0] = sel;
+            sm.misc[1] = want - cum;
+        }
+        bar_sync(BAR, NT);
+        prefix |= (unsigned long long)sm.misc[0] << (8 * pass);
+        mask |= 255ull << (8 * pass);
+        want = sm.misc[1];
+    }
+    const unsigned long long kth = prefix;
+
+    // ---- 5b. ordered lists of holes (< n') and movers (>= n'), then the moves ---------
+    const int n_new = n - k;
+    int32_t* holes = L.list_a + (size_t)u * cap;
+    int32_t* movers = L.list_b + (size_t)u * cap;
+    int hc = 0, mc = 0, ec = 0;
+    for (int base = 0; base < n; base += NT) {
+        const int i = base + tid;
+        const bool valid = i < n;
+        const unsigned long long key = valid ? keys[i] : ~0ull;
+        const bool ev = valid && key <= kth;
+        const bool hole = ev && i < n_new;
+        const bool mover = valid && !ev && i >= n_new;
+        const unsigned bh = __ballot_sync(0xffffffffu, hole);
+        const unsigned bm = __ballot_sync(0xffffffffu, mover);
+        const unsigned be = __ballot_sync(0xffffffffu, ev);
+        const unsigned lt = (1u << lane) - 1u;
+        if (lane == 0) { sm.cnt[0][warp] = __popc(bh); sm.cnt[1][warp] = __popc(bm); sm.cnt[2][warp] = __popc(be); }
+        bar_sync(BAR, NT);
+        int ph = 0, pm = 0, pe = 0, th = 0, tm = 0, te = 0;
+        for (int w2 = 0; w2 < NW; ++w2) {
+            if (w2 < warp) { ph += sm.cnt[0][w2]; pm += sm.cnt[1][w2]; pe += sm.cnt[2][w2]; }
+            th += sm.cnt[0][w2]; tm += sm.cnt[1][w2]; te += sm.cnt[2][w2];
+        }
+        if (hole) holes[hc + ph + __popc(bh & lt)] = i;
+        if (mover) movers[mc + pm + __popc(bm & lt)] = i;
+        if (ev) {
+            const int j = ec + pe + __popc(be & lt);
+            L.ev_pos[(size_t)u * cap + j] = (int32_t)(unsigned)(key & 0xffffffffu);
+            L.ev_score[(size_t)u * cap + j] = __uint_as_float((unsigned)(key >> 32));
+        }
+        hc += th; mc += tm; ec += te;
+        bar_sync(BAR, NT);
+    }
+    if (hc != mc || ec != k) {
+        if (tid == 0) atomicCAS(p.status, kStatusOk, kStatusDeviceCheck);
+    } else {
+        for (int j = warp; j < hc; j += NW) {
+            const int src = movers[j], dst = holes[j];
+            copy_row_swizzled(L.Kd, ubase, rowb, src, dst, lane);
+            copy_row_swizzled(L.Vd, ubase, rowb, src, dst, lane);
+            if (lane == 0) { score[dst] = score[src]; pos[dst] = pos[src]; }
+        }
+    }
+    if (tid == 0) L.ticket[u] = 0;
+}
+
+}  // namespace mkv

@@ -1,0 +1,85 @@
+"""The C-ABI library without a GPU: it loads, exports every declared symbol, its host
+arithmetic is right, and it refuses to run without a device (no fallback)."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+import paper_2605_29873_b200 as mkv
+from paper_2605_29873_b200 import build as mkv_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    mkv_build.build_library()
+    return mkv.load_library()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "mkv.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(mkv_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_symbols()
+    assert len(names) >= 18
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in include/mkv.h but not exported"
+    assert sorted(mkv.EXPORTED_SYMBOLS) == names
+
+
+def test_status_strings(lib):
+    assert mkv.status_string(0) == "ok"
+    assert len({mkv.status_string(i) for i in range(9)}) == 9
+
+
+def test_kv_sizing_matches_the_papers_figure(lib):
+    """Sec. 1: an 8B model's 16-bit KV cache takes exactly 128 KB per token and nearly
+    13 GB for 100K tokens (fixture tests/golden/kv_sizing.txt)."""
+    vals = {}
+    for line in open(os.path.join(ROOT, "tests", "golden", "kv_sizing.txt")):
+        if line.strip() and not line.startswith("#"):
+            k, v = line.split()
+            vals[k] = int(v)
+    per_tok = mkv.kv_bytes_per_token(32, 8, 128, mkv.MKV_BF16)
+    assert per_tok == vals["bytes_per_token"] == 128 * 1024
+    assert round(per_tok * vals["tokens"] / 1e9) == vals["approx_gigabytes"]
+    # the workspace grows by that per cached token (plus < 10 % of split-KV scratch)
+    a = mkv.workspace_bytes(32, 4, 32, 8, 128, 2048, 2048)
+    b = mkv.workspace_bytes(32, 4, 32, 8, 128, 2048, 4096)
+    assert (b - a) // (4 * 2048) >= per_tok
+    assert (b - a) // (4 * 2048) < per_tok * 1.10
+
+
+def test_workspace_bytes_rejects_bad_shapes(lib):
+    ok = mkv.workspace_bytes(1, 1, 4, 1, 64, 64, 64, mkv.MKV_F32)
+    assert ok > 0 and ok % 256 == 0
+    assert mkv.workspace_bytes(1, 1, 5, 2, 64, 64, 64) == 0      # q_heads % kv_heads
+    assert mkv.workspace_bytes(1, 1, 4, 1, 96, 64, 64) == 0      # head_dim
+    assert mkv.workspace_bytes(0, 1, 4, 1, 64, 64, 64) == 0
+    assert mkv.workspace_bytes(1, 1, 4, 1, 64, 0, 64) == 0       # budget >= 1
+    assert mkv.workspace_bytes(1, 1, 64, 1, 64, 64, 64) == 0     # group > 16
+
+
+def test_create_validates_then_fails_loudly_without_a_gpu(lib):
+    import torch
+    ctx = C.c_void_p(0)
+    fake = C.c_void_p(1 << 20)   # aligned, never dereferenced by the argument checks
+    n = mkv.workspace_bytes(1, 1, 4, 1, 64, 64, 64, mkv.MKV_F32)
+    args = lambda **kw: [kw.get("layers", 1), 4, 1, 64, 64, C.c_float(kw.get("beta", 0.9)), 1, 64, mkv.MKV_F32,
+                         kw.get("out", mkv.MKV_F32), 0, 0, 0, kw.get("ws", fake), kw.get("n", n), 0, C.byref(ctx)]
+    assert lib.mkv_create(*args(beta=1.5)) == 1
+    assert lib.mkv_create(*args(out=mkv.MKV_BF16)) == 1           # fp32 cache needs fp32 out
+    assert lib.mkv_create(*args(ws=C.c_void_p(0))) == 1
+    assert lib.mkv_create(*args(ws=C.c_void_p((1 << 20) + 8))) == 4
+    assert lib.mkv_create(*args(n=n - 1)) == 4
+    if not torch.cuda.is_available():
+        assert lib.mkv_create(*args()) == 6                       # MKV_ERR_CUDA: no device, no fallback
+        with pytest.raises(RuntimeError):
+            mkv.MomentKV(1, 4, 1, 64, 64, 0.9, 1, 64, kv_dtype=mkv.MKV_F32)
+    assert lib.mkv_decode_step(None, 0, None, None, None, None, None) == 1
+    lib.mkv_destroy(None)

@@ -110,7 +110,11 @@ class SequenceStream:
         self.Lp = int(w.prefill_lens()[b] if prefill_len is None else prefill_len)
         d = w.head_dim
         self._rng_p = np.random.default_rng([w.seed, layer, b, 0])
+        # one generator per drawn tensor, so that the stream does not depend on how the
+        # steps are split into next() calls
         self._rng_t = np.random.default_rng([w.seed, layer, b, 1])
+        self._rng_k = np.random.default_rng([w.seed, layer, b, 3])
+        self._rng_v = np.random.default_rng([w.seed, layer, b, 4])
         rng_u = np.random.default_rng([w.seed, layer, b, 2])
         # heavy-hitter directions u[g][j][d]
         if w.n_heavy > 0:
@@ -153,8 +157,8 @@ class SequenceStream:
         d, G = w.head_dim, w.group
         sig = np.sqrt(1.0 - w.rho ** 2)
         eps = self._rng_t.standard_normal((n, w.q_heads, d))
-        kk = self._rng_t.standard_normal((n, w.kv_heads, d)) / np.sqrt(d)
-        vv = self._rng_t.standard_normal((n, w.kv_heads, d)) / np.sqrt(d)
+        kk = self._rng_k.standard_normal((n, w.kv_heads, d)) / np.sqrt(d)
+        vv = self._rng_v.standard_normal((n, w.kv_heads, d)) / np.sqrt(d)
         z, _ = lfilter([sig], [1.0, -w.rho], eps, axis=0, zi=(w.rho * self._z)[None])
         self._z = z[-1].copy()
         ts = np.arange(self.t, self.t + n)
