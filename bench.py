@@ -206,12 +206,15 @@ def main():
     ap.add_argument("--config", default="llama_b16", choices=sorted(CONFIGS))
     ap.add_argument("--layers", type=int, default=4)
     ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "mma"])
+    ap.add_argument("--budget", type=int, default=0, help="override the workload's decode budget (profiling small cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     w = CONFIGS[args.config]
+    if args.budget > 0:
+        w = w.with_(budget=args.budget)
     if args.impl == "reference":
         run_reference(args, w)
         return

@@ -18,22 +18,15 @@ namespace {
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
-inline int round16(int a) { return (a + 15) / 16 * 16; }
+inline int round4(int a) { return (a + 3) / 4 * 4; }
 inline int elem_size(int dt) { return dt == MKV_BF16 ? 2 : 4; }
 
-// smallest item size the work list may ever use for this shape: bounds the number of
-// partials per unit (kMaxParts) and therefore the scratch the workspace must hold
-int min_item_rows(int max_prefill, int cap) {
-    const int need = round16(ceil_div(max_prefill + cap, kMaxParts - 2));
-    return std::max(64, need);
-}
-
 struct LayerOff {
-    size_t Kp, Vp, Kd, Vd, score, pos, n_dec, logit, abar, n_prev, ev_k, ev_pos, ev_score, items, unit_lp,
-        unit_part0, unit_nparts, part_o, part_ml, ticket, sched, step, keys, list_a, list_b, end;
+    size_t Kp, Vp, Kd, Vd, score, pos, n_dec, logit, abar, n_prev, ev_k, ev_pos, ev_score, items, cta_item0,
+        unit_lp, unit_part0, unit_nparts, part_o, part_ml, ticket, unit_step, keys, list_a, list_b, end;
 };
 struct Layout {
-    int units, cap, rowb, max_items;
+    int units, cap, rowb, max_items, lstride;
     size_t status, stage_q, stage_k, stage_v, stage_out, layer0, layer_bytes, total;
     LayerOff lo;  // offsets relative to the layer base
 };
@@ -51,8 +44,9 @@ bool make_layout(int layers, int batch, int q_heads, int kv_heads, int head_dim,
     L.units = batch * kv_heads;
     L.cap = budget + 1;
     L.rowb = head_dim * elem_size(kv_dtype);
-    const int irm = min_item_rows(max_prefill, L.cap);
-    L.max_items = L.units * (ceil_div(max_prefill, irm) + ceil_div(L.cap, irm));
+    L.lstride = round4(L.cap);
+    // every CTA range yields one item plus one more per unit boundary it crosses
+    L.max_items = kMaxCtas + L.units;
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes); return r; };
     L.status = take(256);
@@ -70,21 +64,21 @@ bool make_layout(int layers, int batch, int q_heads, int kv_heads, int head_dim,
     L.lo.score = take(U * C * 4);
     L.lo.pos = take(U * C * 4);
     L.lo.n_dec = take(U * 4);
-    L.lo.logit = take((size_t)batch * q_heads * C * 4);
+    L.lo.logit = take((size_t)batch * q_heads * L.lstride * 4);
     L.lo.abar = take(U * C * 4);
     L.lo.n_prev = take(U * 4);
     L.lo.ev_k = take(U * 4);
     L.lo.ev_pos = take(U * C * 4);
     L.lo.ev_score = take(U * C * 4);
     L.lo.items = take((size_t)L.max_items * sizeof(Item));
+    L.lo.cta_item0 = take((size_t)(kMaxCtas + 1) * 4);
     L.lo.unit_lp = take(U * 4);
     L.lo.unit_part0 = take(U * 4);
     L.lo.unit_nparts = take(U * 4);
     L.lo.part_o = take((size_t)L.max_items * G * head_dim * 4);
     L.lo.part_ml = take((size_t)L.max_items * G * 2 * 4);
     L.lo.ticket = take(U * 4);
-    L.lo.sched = take(256);
-    L.lo.step = take(256);
+    L.lo.unit_step = take(U * 4);
     L.lo.keys = take(U * C * 8);
     L.lo.list_a = take(U * C * 4);
     L.lo.list_b = take(U * C * 4);
@@ -127,11 +121,11 @@ struct mkv_ctx {
     int device;
     uint8_t* ws;
     Layout lay;
-    int item_rows;
-    int n_ctas;     // persistent grid of the tensor-core kernel
+    int n_ctas_max; // persistent grid upper bound (SM count x resident CTAs per SM)
     bool use_mma;
     std::vector<char> prefilled;
     std::vector<int> n_items;
+    std::vector<int> n_ctas;
     std::vector<std::vector<int32_t>> lens;   // per layer, per sequence
     int64_t launches;
 };
@@ -153,15 +147,16 @@ LayerDev layer_dev(const mkv_ctx* c, int layer) {
     d.ev_pos = (int32_t*)(base + o.ev_pos);
     d.ev_score = (float*)(base + o.ev_score);
     d.items = (const Item*)(base + o.items);
+    d.cta_item0 = (const int32_t*)(base + o.cta_item0);
     d.n_items = c->n_items[layer];
+    d.n_ctas = c->n_ctas[layer];
     d.unit_lp = (const int32_t*)(base + o.unit_lp);
     d.unit_part0 = (const int32_t*)(base + o.unit_part0);
     d.unit_nparts = (const int32_t*)(base + o.unit_nparts);
     d.part_o = (float*)(base + o.part_o);
     d.part_ml = (float*)(base + o.part_ml);
     d.ticket = (int32_t*)(base + o.ticket);
-    d.sched = (int32_t*)(base + o.sched);
-    d.step = (int32_t*)(base + o.step);
+    d.unit_step = (int32_t*)(base + o.unit_step);
     d.keys = (unsigned long long*)(base + o.keys);
     d.list_a = (int32_t*)(base + o.list_a);
     d.list_b = (int32_t*)(base + o.list_b);
@@ -177,6 +172,7 @@ Params make_params(const mkv_ctx* c, int layer, const void* q, const void* k_new
     p.batch = c->batch; p.q_heads = c->q_heads; p.kv_heads = c->kv_heads; p.group = c->group;
     p.head_dim = c->head_dim;
     p.cap = c->lay.cap; p.max_prefill = c->max_prefill; p.budget = c->budget;
+    p.lstride = c->lay.lstride;
     p.beta = c->beta;
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c->head_dim));
     p.mode = mode;
@@ -185,13 +181,14 @@ Params make_params(const mkv_ctx* c, int layer, const void* q, const void* k_new
 }
 
 mkv_status launch_step(mkv_ctx* c, const Params& p, cudaStream_t st) {
-    cudaError_t e = c->use_mma ? launch_mma(p, c->n_ctas, st) : launch_simt(p, c->kv_dtype, st);
+    cudaError_t e = c->use_mma ? launch_mma(p, st) : launch_simt(p, c->kv_dtype, st);
     if (e != cudaSuccess) return MKV_ERR_CUDA;
     c->launches += 1;
     return MKV_OK;
 }
 
 bool layer_ok(const mkv_ctx* c, int layer) { return c && layer >= 0 && layer < c->layers; }
+bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
 struct DeviceGuard {
     int prev = -1; bool ok;
@@ -262,14 +259,12 @@ mkv_status mkv_create(int layers, int q_heads, int kv_heads, int head_dim, int b
     c->kv_dtype = kv_dtype; c->out_dtype = out_dtype; c->score_mode = score_mode; c->kernel = kernel;
     c->flags = flags; c->device = device; c->ws = (uint8_t*)workspace; c->lay = L;
     c->use_mma = use_mma;
-    int ir = 256;
-    if (const char* e = std::getenv("MKV_ITEM_ROWS")) ir = std::atoi(e);
-    c->item_rows = std::max(min_item_rows(max_prefill, L.cap), round16(std::max(ir, 16)));
-    int per_sm = 2;
-    if (const char* e = std::getenv("MKV_CTAS_PER_SM")) per_sm = std::max(1, std::min(4, std::atoi(e)));
-    c->n_ctas = prop.multiProcessorCount * per_sm;
+    int per_sm = use_mma ? 2 : 8;
+    if (const char* e = std::getenv("MKV_CTAS_PER_SM")) per_sm = std::max(1, std::min(16, std::atoi(e)));
+    c->n_ctas_max = std::min(kMaxCtas, prop.multiProcessorCount * per_sm);
     c->prefilled.assign(layers, 0);
     c->n_items.assign(layers, 0);
+    c->n_ctas.assign(layers, 0);
     c->lens.assign(layers, std::vector<int32_t>(batch, 0));
     c->launches = 0;
     *out_ctx = c;
@@ -292,33 +287,61 @@ mkv_status mkv_prefill(mkv_ctx* c, int layer, const void* K, const void* V, cons
     if (!guard.ok) return MKV_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;
     const Layout& L = c->lay;
-    const int U = L.units, cap = L.cap, ir = c->item_rows;
+    const int U = L.units;
 
-    // static work list: unit-major, prefill segment then decode segment, pieces of equal
-    // size (a multiple of 16 rows) no longer than item_rows
-    std::vector<Item> items;
-    std::vector<int32_t> lp(U), part0(U), nparts(U);
+    // Static work list.  A unit's rows are a sequence of 64-row tiles (prefill tiles, then
+    // the decode tiles of the budget's row range); all units' tiles laid end to end are cut
+    // into equally long contiguous ranges, one per CTA; a range that crosses a unit
+    // boundary splits into items.  Ranges are long enough to keep a unit's item count
+    // within kMaxParts.
+    const int td = ceil_div(c->budget_max, kTileRows);
+    std::vector<int32_t> lp(U), part0(U), nparts(U, 0);
+    std::vector<long long> tile_begin(U + 1, 0);
+    int max_unit_tiles = 1;
     for (int u = 0; u < U; ++u) {
-        const int len = prefill_lens[u / c->kv_heads];
-        lp[u] = len;
-        part0[u] = (int32_t)items.size();
-        for (int seg = 0; seg < 2; ++seg) {
-            const int total = seg == 0 ? len : cap;
-            if (total == 0) continue;
-            const int pieces = ceil_div(total, ir);
-            const int piece = round16(ceil_div(total, pieces));
-            for (int r0 = 0; r0 < total; r0 += piece) items.push_back(Item{u, r0, std::min(piece, total - r0), seg});
-        }
-        nparts[u] = (int32_t)items.size() - part0[u];
-        if (nparts[u] > kMaxParts) return MKV_ERR_CAPACITY;
+        lp[u] = prefill_lens[u / c->kv_heads];
+        const int tu = ceil_div(lp[u], kTileRows) + td;
+        tile_begin[u + 1] = tile_begin[u] + tu;
+        max_unit_tiles = std::max(max_unit_tiles, tu);
     }
-    if ((int)items.size() > L.max_items) return MKV_ERR_CAPACITY;
+    const long long t_all = tile_begin[U];
+    long long per_cta = std::max<long long>(ceil_div(max_unit_tiles, kMaxParts / 2 - 4), (t_all + c->n_ctas_max - 1) / c->n_ctas_max);
+    const int n_ctas = (int)((t_all + per_cta - 1) / per_cta);
+    std::vector<Item> items;
+    std::vector<int32_t> cta_item0(n_ctas + 1, 0);
+    {
+        int u = 0;
+        for (int cta = 0; cta < n_ctas; ++cta) {
+            cta_item0[cta] = (int32_t)items.size();
+            long long t0 = t_all * cta / n_ctas;
+            const long long t1 = t_all * (cta + 1) / n_ctas;
+            while (t0 < t1) {
+                while (tile_begin[u + 1] <= t0) ++u;
+                const long long e = std::min(t1, tile_begin[u + 1]);
+                items.push_back(Item{u, (int32_t)(t0 - tile_begin[u]), (int32_t)(e - t0), 0});
+                nparts[u] += 1;
+                t0 = e;
+            }
+        }
+        cta_item0[n_ctas] = (int32_t)items.size();
+    }
+    // partial index = item index; a unit's items are consecutive because ranges are in order
+    {
+        std::vector<char> seen(U, 0);
+        for (size_t i = 0; i < items.size(); ++i)
+            if (!seen[items[i].unit]) { seen[items[i].unit] = 1; part0[items[i].unit] = (int32_t)i; }
+    }
+    for (int u = 0; u < U; ++u)
+        if (nparts[u] < 1 || nparts[u] > kMaxParts) return MKV_ERR_CAPACITY;
+    if ((int)items.size() > L.max_items || n_ctas > kMaxCtas) return MKV_ERR_CAPACITY;
     c->n_items[layer] = (int)items.size();
+    c->n_ctas[layer] = n_ctas;
     for (int b = 0; b < c->batch; ++b) c->lens[layer][b] = prefill_lens[b];
 
     uint8_t* base = c->ws + L.layer0 + L.layer_bytes * (size_t)layer;
     bool ok = true;
     ok &= cudaMemcpyAsync(base + L.lo.items, items.data(), items.size() * sizeof(Item), cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(base + L.lo.cta_item0, cta_item0.data(), cta_item0.size() * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok &= cudaMemcpyAsync(base + L.lo.unit_lp, lp.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok &= cudaMemcpyAsync(base + L.lo.unit_part0, part0.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok &= cudaMemcpyAsync(base + L.lo.unit_nparts, nparts.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
@@ -327,8 +350,7 @@ mkv_status mkv_prefill(mkv_ctx* c, int layer, const void* K, const void* V, cons
     ok &= cudaMemsetAsync(base + L.lo.n_prev, 0, U * 4, st) == cudaSuccess;
     ok &= cudaMemsetAsync(base + L.lo.ev_k, 0, U * 4, st) == cudaSuccess;
     ok &= cudaMemsetAsync(base + L.lo.ticket, 0, U * 4, st) == cudaSuccess;
-    ok &= cudaMemsetAsync(base + L.lo.sched, 0, 256, st) == cudaSuccess;
-    ok &= cudaMemsetAsync(base + L.lo.step, 0, 256, st) == cudaSuccess;
+    ok &= cudaMemsetAsync(base + L.lo.unit_step, 0, U * 4, st) == cudaSuccess;
     if (!ok) return MKV_ERR_CUDA;
     // host vectors above are pageable: the runtime has staged them before returning
     if (maxlen > 0) {
@@ -348,6 +370,7 @@ mkv_status mkv_prefill(mkv_ctx* c, int layer, const void* K, const void* V, cons
 mkv_status mkv_decode_step(mkv_ctx* c, int layer, const void* q, const void* k_new, const void* v_new, void* out,
                            void* stream) {
     if (!layer_ok(c, layer) || !q || !k_new || !v_new || !out) return MKV_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out)) return MKV_ERR_INVALID_ARG;
     if (!c->prefilled[layer]) return MKV_ERR_BAD_STATE;
     DeviceGuard guard(c->device);
     if (!guard.ok) return MKV_ERR_CUDA;
@@ -378,6 +401,7 @@ mkv_status mkv_decode_step_host(mkv_ctx* c, int layer, const void* qh, const voi
 
 mkv_status mkv_attend_only(mkv_ctx* c, int layer, const void* q, void* out, void* stream) {
     if (!layer_ok(c, layer) || !q || !out) return MKV_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out)) return MKV_ERR_INVALID_ARG;
     if (!c->prefilled[layer]) return MKV_ERR_BAD_STATE;
     DeviceGuard guard(c->device);
     if (!guard.ok) return MKV_ERR_CUDA;
@@ -502,7 +526,7 @@ mkv_status mkv_get_step(mkv_ctx* c, int layer, int64_t* step) {
     DeviceGuard guard(c->device);
     if (!guard.ok || cudaDeviceSynchronize() != cudaSuccess) return MKV_ERR_CUDA;
     int32_t s = 0;
-    MKV_D2H(&s, layer_dev(c, layer).step, 4);
+    MKV_D2H(&s, layer_dev(c, layer).unit_step, 4);
     *step = s;
     return MKV_OK;
 }

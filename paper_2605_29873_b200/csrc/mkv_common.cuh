@@ -6,8 +6,7 @@
 //   head), so a unit is the granule of scoring, selection and compaction.
 //
 //   Kp, Vp  [units][max_prefill][ROWB]   frozen prefill pool (Sec. 4.2 "Prefill pool")
-//   Kd, Vd  [units][cap][ROWB]           decode pool, cap = largest budget + 1 (the fresh
-//                                        token sits in the pool during its own step)
+//   Kd, Vd  [units][cap][ROWB]           decode pool, cap = largest budget + 1
 //   score   [units][cap] f32             importance I_i (Eq. 5)
 //   pos     [units][cap] i32             decode-step id at which the token was appended
 //   n_dec   [units] i32                  tokens currently in the decode pool
@@ -19,12 +18,18 @@
 // what makes the ldmatrix reads of the tensor-core kernel conflict-free without any
 // per-element shuffling on the way in.
 //
-// Work decomposition: the rows of every unit (prefill segment, then decode segment up to
-// cap) are cut into "items" of at most item_rows rows; an item never straddles the two
-// segments.  An item yields one partial (m, l, O[G][d]) of the online softmax.  The last
-// CTA to deliver a partial of a unit (an atomic ticket, never a wait) runs that unit's
-// tail: combine, normalise the decode probabilities, head mean, momentum update,
-// selection, compaction.
+// Work decomposition.  The rows of a unit form a sequence of 64-row tiles: the prefill
+// tiles, then the decode tiles (over the budget's row range).  All tiles of all units,
+// laid end to end, are cut into one contiguous, equally long range per CTA; where a
+// range crosses a unit boundary it splits into "items".  An item (unit, first tile,
+// tile count) carries one online-softmax state across its tiles and yields one partial
+// (m, l, O[G][d]).  Whoever delivers the last partial of a unit (an atomic ticket, never
+// a wait) runs that unit's tail: the fresh token, combine, normalised decode
+// probabilities, head mean, momentum update, selection, append/compaction.
+//
+// The fresh token of a step never travels through the streaming part: its logit, its
+// probability, its importance and its row store all happen in the tail, which knows the
+// evicted slot by then and writes the fresh row straight into the hole.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -32,8 +37,10 @@
 
 namespace mkv {
 
-constexpr int kMaxGroup = 16;       // G = q_heads / kv_heads
-constexpr int kMaxParts = 128;      // partials per unit (item_rows grows to keep this)
+constexpr int kTileRows = 64;       // rows of one tile of the work decomposition
+constexpr int kMaxGroup = 8;        // G = q_heads / kv_heads the kernels are built for
+constexpr int kMaxParts = 128;      // partials per unit (CTA ranges grow to keep this)
+constexpr int kMaxCtas = 2048;      // persistent grid upper bound (sizes the partial scratch)
 constexpr float kNegBig = -1.0e30f; // finite stand-in for -inf in running maxima
 
 enum : int { kModeDecode = 0, kModeAttendOnly = 1 };
@@ -41,9 +48,9 @@ enum : int { kStatusOk = 0, kStatusTimeout = 7, kStatusDeviceCheck = 8 };
 
 struct Item {          // 16 bytes, read as one int4
     int32_t unit;
-    int32_t row0;      // first row inside the segment
-    int32_t rows;      // rows covered (decode segment: of the capacity range)
-    int32_t seg;       // 0 prefill, 1 decode
+    int32_t tile0;     // first tile inside the unit's tile sequence (prefill tiles first)
+    int32_t ntiles;
+    int32_t pad;
 };
 
 struct LayerDev {
@@ -51,22 +58,23 @@ struct LayerDev {
     float* score;
     int32_t* pos;
     int32_t* n_dec;
-    float* logit;      // [batch*q_heads][cap] raw logits (log2 units) of decode tokens
+    float* logit;      // [batch*q_heads][lstride] raw logits (log2 units) of decode-pool tokens
     float* abar;       // [units][cap] or nullptr
-    int32_t* n_prev;   // [units] decode count before the last eviction
+    int32_t* n_prev;   // [units] decode count (fresh token included) before the last eviction
     int32_t* ev_k;     // [units] tokens evicted by the last step
     int32_t* ev_pos;   // [units][cap]
     float* ev_score;   // [units][cap]
-    const Item* items;
+    const Item* items;          // all items, CTA-major
+    const int32_t* cta_item0;   // [n_ctas + 1] first item of every CTA
     int32_t n_items;
+    int32_t n_ctas;             // CTAs the work list was cut for (= the grid)
     const int32_t* unit_lp;     // [units] prefill length
-    const int32_t* unit_part0;  // [units] first item (= partial) index of the unit
+    const int32_t* unit_part0;  // [units] first partial index of the unit
     const int32_t* unit_nparts; // [units]
     float* part_o;     // [n_items][G][d]
     float* part_ml;    // [n_items][G][2]  (running max in log2 units, running sum)
     int32_t* ticket;   // [units]
-    int32_t* sched;    // [0] work counter  [1] CTAs done
-    int32_t* step;     // [1] decode steps completed
+    int32_t* unit_step;// [units] decode steps completed
     unsigned long long* keys;   // [units][cap] selection scratch
     int32_t* list_a;   // [units][cap] compaction scratch (holes)
     int32_t* list_b;   // [units][cap] compaction scratch (movers)
@@ -81,6 +89,7 @@ struct Params {
     int32_t* status;
     int batch, q_heads, kv_heads, group, head_dim;
     int cap, max_prefill, budget;
+    int lstride;       // floats per head row of the logit scratch (cap rounded up to 4)
     float beta;
     float scale_log2;  // log2(e) / sqrt(head_dim)
     int mode;
@@ -105,16 +114,15 @@ __device__ inline void bar_sync(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
-// Last CTA out of the kernel rewinds the scheduler words and advances the step counter.
-__device__ inline void grid_epilogue(const Params& p, unsigned n_ctas) {
-    __threadfence();
-    const int prev = atomicAdd(&p.L.sched[1], 1);
-    if (prev == (int)n_ctas - 1) {
-        p.L.sched[0] = 0;
-        p.L.sched[1] = 0;
-        if (p.mode == kModeDecode) p.L.step[0] = p.L.step[0] + 1;
-        __threadfence();
-    }
+// Tile `t` of a unit's tile sequence -> (segment, first row, valid rows).  Prefill tiles
+// come first; decode tiles cover the pool's rows [0, n_old).
+struct TileRef { int seg, row, cnt; };
+__device__ inline TileRef tile_ref(int t, int lp, int n_old) {
+    const int tp = (lp + kTileRows - 1) / kTileRows;
+    TileRef r;
+    if (t < tp) { r.seg = 0; r.row = t * kTileRows; r.cnt = min(kTileRows, lp - r.row); }
+    else { r.seg = 1; r.row = (t - tp) * kTileRows; r.cnt = max(0, min(kTileRows, n_old - r.row)); }
+    return r;
 }
 
 }  // namespace mkv

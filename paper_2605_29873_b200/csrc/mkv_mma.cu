@@ -2,27 +2,37 @@
 // path of the Llama-3.1-8B- and Qwen2.5-7B-shaped workloads.
 //
 // Decode attention at GQA group 4-7 is bound by streaming K and V from HBM once per KV
-// head; the kernel is built around that stream.
-//   * Persistent CTAs (two per SM) pull items from an atomic work counter, so the grid is
-//     a multiple of the SM count and load balance does not depend on sequence lengths.
-//   * One producer thread per CTA issues bulk asynchronous copies (the non-tensor TMA
-//     form, no multicast) of 64-row K and V tiles, 16 KB each, into a ring of shared
-//     memory stages; completion is signalled on an mbarrier (complete_tx).  The cache
-//     rows are already chunk-permuted in HBM, so a straight copy lands a layout that
-//     ldmatrix reads without bank conflicts.  The producer keeps prefetching across item
-//     boundaries and while the consumers run a unit's tail.
-//   * Four consumer warps each own 16 rows of a tile.  S = Q K^T and O += P V use
-//     mma.sync m16n8k16 (bf16 in, fp32 accumulate) with the G query heads padded to the
-//     16-row M dimension: this is not a GEMM reshaping for the sake of tensor cores, it
-//     takes the per-row instruction count from ~60 (scalar FMA + shuffles) to ~7 so that
-//     issue slots never limit the HBM stream, for G = 7 as well as G = 4.  The softmax
-//     runs in registers in fp32 (quad shuffles for the row maximum); P enters the second
-//     mma as hi + lo bf16 halves, so the rounding of P to bf16 does not reach `out`.
-//   * Raw fp32 logits of decode-pool tokens are stored (4 bytes per head and token) for
+// head; the kernel is built around that stream.  A CTA is three kinds of warps:
+//
+//   * one PRODUCER thread walks the CTA's items of the static work list (a contiguous,
+//     equally long range of 64-row tiles per CTA) and issues bulk asynchronous copies (the
+//     non-tensor TMA form, no multicast) of K and V tiles, 16 KB each, into a ring of
+//     shared-memory stages; completion is signalled on an mbarrier (complete_tx).  The
+//     cache rows are already chunk-permuted in HBM, so a straight copy lands a layout that
+//     ldmatrix reads without bank conflicts.  The first tile of an item also brings the
+//     unit's G query rows.  The producer runs ahead across item boundaries.
+//   * four CONSUMER warps each own 16 rows of a tile and never synchronise with one
+//     another.  S = Q K^T uses mma.sync m16n8k16 (bf16 in, fp32 accumulate) with the G
+//     query heads in the M dimension; its accumulator fragment is, register for register,
+//     the B operand of the transposed second product O^T += V^T P^T (head_dim in M, the
+//     heads in N = 8), so P never leaves the registers and no work is spent on padding
+//     rows.  This is not a GEMM reshaping for the sake of tensor cores: it takes the
+//     per-row instruction count from ~60 (scalar FMA + shuffles) to ~4 so that issue slots
+//     never limit the HBM stream, for G = 7 as well as G = 4.  The softmax runs in
+//     registers in fp32 (quad shuffles for the row maximum); P enters the second mma as
+//     hi + lo bf16 halves, so the rounding of P to bf16 does not reach `out`.
+//     Raw fp32 logits of decode-pool tokens are stored (4 bytes per head and token) for
 //     the tail, which needs the global log-sum-exp before it can normalise them (Eq. 4).
-//   * At the end of an item the four warps merge (m, l, O) through shared memory, write
-//     one partial and take the unit's ticket; the last ticket holder runs the tail.
-// Every wait is bounded: on expiry the kernel records MKV_ERR_TIMEOUT and drains.
+//   * four TAIL warps.  At the end of an item the consumers drop their (m, l, O) into a
+//     ring stage borrowed from the producer and go straight on to the next item; the tail
+//     warps merge the four states into one partial in global memory, take the unit's
+//     ticket and, when it is the last one, run the unit's tail (fresh token, combine,
+//     probabilities, momentum update, selection, append/compaction) while the stream
+//     continues.
+// Every wait is bounded: on expiry the kernel records MKV_ERR_TIMEOUT, every role drains
+// (the producer waits, bounded again, for its copies in flight) and the CTA returns.
+#include <cstdlib>
+
 #include "mkv_launch.h"
 #include "mkv_ptx.cuh"
 #include "mkv_tail.cuh"
@@ -30,78 +40,93 @@
 namespace mkv {
 namespace {
 
-constexpr int kTileRows = 64;
 constexpr int kRowB = 256;                                // 128 bf16
 constexpr int kTileBytes = kTileRows * kRowB;             // 16 KB (K or V)
 constexpr int kStageBytes = 2 * kTileBytes;               // K then V
+constexpr int kQSlotBytes = kMaxGroup * kRowB;            // query rows of one unit
 constexpr int kConsumerWarps = 4;
+constexpr int kTailWarps = 4;
 constexpr int kConsumers = kConsumerWarps * 32;
-constexpr int kThreads = kConsumers + 32;
+constexpr int kTailThreads = kTailWarps * 32;
+constexpr int kTailTid0 = kConsumers + 32;                // first thread of the tail group
+constexpr int kThreads = kConsumers + 32 + kTailThreads;
 constexpr int kMaxStages = 8;
-constexpr unsigned long long kWaitNs = 4000000000ull;     // 4 s
+constexpr int kXoStride = 132;                            // floats per head row of the exchange
+constexpr unsigned long long kWaitNs = 2000000000ull;     // 2 s
+
+enum : int { kEntryTile = 0, kEntryExchange = 1, kEntryEnd = 2 };
 
 struct StageMeta {
-    int item;       // -1: no more work
+    int kind;
     int unit;
-    int seg;
-    int row;        // slot of the tile's first row inside its pool (multiple of 16)
-    int cnt_pool;   // rows copied from the pool
-    int fresh_row;  // tile row that takes the step's fresh token, or -1
-    int first, last;
+    int item;
+    int seg;        // 0 prefill, 1 decode
+    int row;        // slot of the tile's first row inside its pool (multiple of 64)
+    int cnt;        // valid rows
+    int first;      // first entry of its item: reset the running state
+    int pad;
 };
 
-template <int GR>
-struct MergeSmem {
-    static constexpr int NH = GR / 4;          // column halves merged one after the other
-    static constexpr int HC = 128 / NH;
-    float xm[kConsumerWarps][GR];
-    float xl[kConsumerWarps][GR];
-    float xo[kConsumerWarps][GR][HC + 4];
-};
-
-template <int GR>
-union alignas(16) ScratchSmem {
-    TailSmem<kConsumers> tail;
-    MergeSmem<GR> merge;
-};
+struct ExchangeRef { int stage, unit, item, pad; };
 
 struct Control {
     unsigned long long full[kMaxStages];
     unsigned long long empty[kMaxStages];
+    unsigned long long xfull[kMaxStages];
     StageMeta meta[kMaxStages];
+    ExchangeRef xq[kMaxStages];
     int abort_flag;
     int last_flag;
+    int wait_ok;
 };
 
-template <int GR>
 constexpr size_t smem_bytes(int nst) {
-    return (size_t)nst * kStageBytes + sizeof(ScratchSmem<GR>) + sizeof(Control);
+    return (size_t)nst * (kStageBytes + kQSlotBytes) + sizeof(TailSmem<kTailThreads>) + sizeof(Control) + 64;
 }
+
+__device__ inline bool aborted(const Control* ctl) { return *reinterpret_cast<const volatile int*>(&ctl->abort_flag) != 0; }
 
 __device__ inline void note_timeout(const Params& p, Control* ctl) {
     atomicCAS(p.status, kStatusOk, kStatusTimeout);
     *reinterpret_cast<volatile int*>(&ctl->abort_flag) = 1;
 }
 
-template <int GR>
+// Bounded mbarrier wait that also gives up as soon as another role has aborted.
+__device__ inline bool wait_or_abort(uint32_t bar, uint32_t parity, Control* ctl) {
+    for (int i = 0; i < 32; ++i)
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = ptx::globaltimer_ns();
+    for (;;) {
+        for (int i = 0; i < 128; ++i)
+            if (ptx::mbar_try_wait(bar, parity)) return true;
+        if (aborted(ctl)) return false;
+        if (ptx::globaltimer_ns() - t0 > kWaitNs) return false;
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const int nst) {
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t* const stages = smem;
-    ScratchSmem<GR>* const scratch = reinterpret_cast<ScratchSmem<GR>*>(smem + (size_t)nst * kStageBytes);
-    Control* const ctl = reinterpret_cast<Control*>(smem + (size_t)nst * kStageBytes + sizeof(ScratchSmem<GR>));
+    uint8_t* const qslots = smem + (size_t)nst * kStageBytes;
+    TailSmem<kTailThreads>* const tsm =
+        reinterpret_cast<TailSmem<kTailThreads>*>(qslots + (size_t)nst * kQSlotBytes);
+    Control* const ctl = reinterpret_cast<Control*>(reinterpret_cast<uint8_t*>(tsm) + ((sizeof(TailSmem<kTailThreads>) + 15) & ~size_t(15)));
 
     const LayerDev& L = p.L;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool dec = (p.mode == kModeDecode);
     const int G = p.group;
+    const int item_begin = L.cta_item0[blockIdx.x], item_end = L.cta_item0[blockIdx.x + 1];
 
     if (tid == 0) {
         for (int s = 0; s < nst; ++s) {
             ptx::mbar_init(ptx::smem_u32(&ctl->full[s]), 1);
             ptx::mbar_init(ptx::smem_u32(&ctl->empty[s]), kConsumerWarps);
+            ptx::mbar_init(ptx::smem_u32(&ctl->xfull[s]), kConsumerWarps);
         }
         ctl->abort_flag = 0;
         ctl->last_flag = 0;
+        ctl->wait_ok = 1;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async();
     }
@@ -112,242 +137,266 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
+            uint32_t issued = 0;       // bit s: a copy into stage s may still be in flight
+            uint32_t issued_par = 0;   // parity its full barrier completes with
             bool ok = true;
-            while (ok) {
-                const int it = atomicAdd(&L.sched[0], 1);
-                if (it >= L.n_items) break;
+            auto acquire = [&]() -> bool {
+                if (!wait_or_abort(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl)) {
+                    if (!aborted(ctl)) note_timeout(p, ctl);
+                    return false;
+                }
+                issued &= ~(1u << stage);
+                return true;
+            };
+            auto advance = [&]() { if (++stage == nst) { stage = 0; phase ^= 1u; } };
+            for (int it = item_begin; it < item_end && ok; ++it) {
                 const int4 v = __ldg(reinterpret_cast<const int4*>(&L.items[it]));
-                const int u = v.x, row0 = v.y, rows = v.z, seg = v.w;
-                int pool_rows, fresh = -1;
-                const uint8_t *kb, *vb;
-                if (seg == 0) {
-                    pool_rows = rows;
-                    kb = L.Kp + ((size_t)u * p.max_prefill + row0) * kRowB;
-                    vb = L.Vp + ((size_t)u * p.max_prefill + row0) * kRowB;
-                } else {
-                    const int n_old = min(L.n_dec[u], p.cap - (dec ? 1 : 0));
-                    pool_rows = max(0, min(rows, n_old - row0));
-                    if (dec && n_old >= row0 && n_old < row0 + rows) fresh = n_old - row0;
-                    kb = L.Kd + ((size_t)u * p.cap + row0) * kRowB;
-                    vb = L.Vd + ((size_t)u * p.cap + row0) * kRowB;
-                }
-                const int total = pool_rows + (fresh >= 0 ? 1 : 0);
-                const int ntiles = max(1, (total + kTileRows - 1) / kTileRows);
-                for (int t = 0; t < ntiles; ++t) {
-                    const uint32_t fb = ptx::smem_u32(&ctl->full[stage]);
-                    if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, kWaitNs)) {
-                        note_timeout(p, ctl);
-                        ok = false;
-                        break;
-                    }
-                    if (*reinterpret_cast<volatile int*>(&ctl->abort_flag)) { ok = false; break; }
-                    const int r = t * kTileRows;
-                    const int cnt = max(0, min(kTileRows, pool_rows - r));
+                const int u = v.x, tile0 = v.y, ntiles = v.z;
+                const int lp = L.unit_lp[u];
+                const int n_old = min(L.n_dec[u], p.cap - (dec ? 1 : 0));
+                const int b = u / p.kv_heads, g = u - b * p.kv_heads;
+                int first = 1;
+                for (int t = tile0; t < tile0 + ntiles; ++t) {
+                    const TileRef tr = tile_ref(t, lp, n_old);
+                    if (tr.cnt == 0) continue;
+                    if (!(ok = acquire())) break;
                     StageMeta& mt = ctl->meta[stage];
-                    mt.item = it; mt.unit = u; mt.seg = seg; mt.row = row0 + r; mt.cnt_pool = cnt;
-                    mt.fresh_row = (fresh >= r && fresh < r + kTileRows) ? fresh - r : -1;
-                    mt.first = (t == 0); mt.last = (t == ntiles - 1);
-                    if (cnt > 0) {
-                        const uint32_t dstK = ptx::smem_u32(stages + (size_t)stage * kStageBytes);
-                        ptx::mbar_arrive_expect_tx(fb, (uint32_t)cnt * 2u * kRowB);
-                        ptx::bulk_g2s(dstK, kb + (size_t)r * kRowB, (uint32_t)cnt * kRowB, fb);
-                        ptx::bulk_g2s(dstK + kTileBytes, vb + (size_t)r * kRowB, (uint32_t)cnt * kRowB, fb);
-                    } else {
-                        ptx::mbar_arrive(fb);
+                    mt.kind = kEntryTile; mt.unit = u; mt.item = it; mt.seg = tr.seg; mt.row = tr.row;
+                    mt.cnt = tr.cnt; mt.first = first;
+                    const uint32_t fb = ptx::smem_u32(&ctl->full[stage]);
+                    const uint32_t dstK = ptx::smem_u32(stages + (size_t)stage * kStageBytes);
+                    const size_t off = ((size_t)u * (tr.seg == 0 ? p.max_prefill : p.cap) + tr.row) * kRowB;
+                    const uint8_t* kb = (tr.seg == 0 ? L.Kp : L.Kd) + off;
+                    const uint8_t* vb = (tr.seg == 0 ? L.Vp : L.Vd) + off;
+                    const uint32_t bytes = (uint32_t)tr.cnt * kRowB;
+                    ptx::mbar_arrive_expect_tx(fb, 2u * bytes + (first ? (uint32_t)G * kRowB : 0u));
+                    ptx::bulk_g2s(dstK, kb, bytes, fb);
+                    ptx::bulk_g2s(dstK + kTileBytes, vb, bytes, fb);
+                    if (first) {
+                        const uint8_t* qsrc = reinterpret_cast<const uint8_t*>(p.q) +
+                                              ((size_t)b * p.q_heads + (size_t)g * G) * kRowB;
+                        ptx::bulk_g2s(ptx::smem_u32(qslots + (size_t)stage * kQSlotBytes), qsrc, (uint32_t)G * kRowB, fb);
                     }
-                    if (++stage == nst) { stage = 0; phase ^= 1u; }
+                    issued |= 1u << stage;
+                    issued_par = (issued_par & ~(1u << stage)) | (phase << stage);
+                    first = 0;
+                    advance();
                 }
+                if (!ok) break;
+                // the item's exchange entry: the consumers hand their state to the tail warps
+                if (!(ok = acquire())) break;
+                StageMeta& mt = ctl->meta[stage];
+                mt.kind = kEntryExchange; mt.unit = u; mt.item = it; mt.seg = 0; mt.row = 0; mt.cnt = 0; mt.first = first;
+                ptx::mbar_arrive(ptx::smem_u32(&ctl->full[stage]));
+                advance();
             }
-            if (ok) {
-                if (ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, kWaitNs)) {
-                    ctl->meta[stage].item = -1;
-                    ptx::mbar_arrive(ptx::smem_u32(&ctl->full[stage]));
-                } else {
-                    note_timeout(p, ctl);
-                }
+            if (ok && acquire()) {
+                ctl->meta[stage].kind = kEntryEnd;
+                ptx::mbar_arrive(ptx::smem_u32(&ctl->full[stage]));
+            } else {
+                // abort: leave only after every copy this thread issued has landed
+                for (int s = 0; s < nst; ++s)
+                    if (issued & (1u << s))
+                        wait_or_abort(ptx::smem_u32(&ctl->full[s]), (issued_par >> s) & 1u, ctl) ||
+                            ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->full[s]), (issued_par >> s) & 1u, kWaitNs);
             }
         }
         __syncwarp();
-    } else {
+    } else if (warp < kConsumerWarps) {
         // ================================ consumers ====================================
         int stage = 0;
         uint32_t phase = 0;
-        float oacc[16][4];
+        int xcount = 0;
+        float oacc[8][4];              // O^T: [16-dim block][dim 0-7 | 8-15 x head pair]
         float m_run = kNegBig, l_run = 0.f;
         uint32_t qa[8][2];
         const int head = lane >> 2, tk0 = 2 * (lane & 3);
         const int mi = lane >> 3, rr = lane & 7;
         const int blk0 = warp * 16;
+        float* lg = L.logit;           // this lane's head row of the unit's logit scratch
 #pragma unroll
-        for (int j = 0; j < 16; ++j) { oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f; }
+        for (int j = 0; j < 8; ++j) { oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f; }
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) { qa[ks][0] = qa[ks][1] = 0u; }
 
         for (;;) {
-            if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->full[stage]), phase, kWaitNs)) {
-                if (lane == 0) note_timeout(p, ctl);
+            if (!wait_or_abort(ptx::smem_u32(&ctl->full[stage]), phase, ctl)) {
+                if (lane == 0 && !aborted(ctl)) note_timeout(p, ctl);
                 break;
             }
             const StageMeta mt = ctl->meta[stage];
-            if (mt.item < 0) break;
-            const int u = mt.unit;
-            const int b = u / p.kv_heads, g = u - b * p.kv_heads;
-            if (mt.first) {
-                const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(p.q) +
-                                            ((size_t)b * p.q_heads + (size_t)g * G + min(head, G - 1)) * 128 + tk0;
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t x0 = __ldg(reinterpret_cast<const uint32_t*>(qrow + 16 * ks));
-                    const uint32_t x1 = __ldg(reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8));
-                    qa[ks][0] = head < G ? x0 : 0u;
-                    qa[ks][1] = head < G ? x1 : 0u;
-                }
-                m_run = kNegBig; l_run = 0.f;
-#pragma unroll
-                for (int j = 0; j < 16; ++j) { oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f; }
-            }
+            if (mt.kind == kEntryEnd) break;
             uint8_t* const sK = stages + (size_t)stage * kStageBytes;
             uint8_t* const sV = sK + kTileBytes;
-            const int nv = mt.cnt_pool + (mt.fresh_row >= 0 ? 1 : 0);
-            bool wrote = false;
-            if (mt.fresh_row >= 0 && (mt.fresh_row >> 4) == warp) {
-                // Algorithm 1 append: the fresh token joins the tile from k_new / v_new and is
-                // stored into its pool slot for the following steps.
-                const int c = lane & 15;
-                const bool isv = lane >= 16;
-                const uint4 val = *reinterpret_cast<const uint4*>(
-                    reinterpret_cast<const uint8_t*>(isv ? p.v_new : p.k_new) + (size_t)u * kRowB + c * 16);
-                const int fr = mt.fresh_row;
-                const uint32_t off = (uint32_t)fr * kRowB + (uint32_t)((c ^ (fr & 7)) << 4);
-                *reinterpret_cast<uint4*>((isv ? sV : sK) + off) = val;
-                const int slot = mt.row + fr;
-                *reinterpret_cast<uint4*>((isv ? L.Vd : L.Kd) + ((size_t)u * p.cap + slot) * kRowB +
-                                          (uint32_t)((c ^ (slot & 7)) << 4)) = val;
-                wrote = true;
-            }
-            if (nv > blk0 && nv < blk0 + 16) {
-                // rows past the valid ones enter the second mma with probability 0: their V
-                // bytes must be finite, so clear them (stale shared memory may hold anything)
-                const int nz = (blk0 + 16 - nv) * 16;
-                for (int idx = lane; idx < nz; idx += 32)
-                    *reinterpret_cast<uint4*>(sV + (size_t)(nv + (idx >> 4)) * kRowB + ((idx & 15) << 4)) =
-                        make_uint4(0u, 0u, 0u, 0u);
-                wrote = true;
-            }
-            __syncwarp();
-
-            if (nv > blk0) {
-                // ---------------- S = Q K^T for 16 heads (padded) x 16 tokens ----------------
-                float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-                const uint32_t kbase = ptx::smem_u32(sK) + (uint32_t)(blk0 + (mi >> 1) * 8 + rr) * kRowB;
+            if (mt.first) {
+                m_run = kNegBig; l_run = 0.f;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    uint32_t b00, b01, b10, b11;
-                    ptx::ldmatrix_x4(kbase + (uint32_t)(((2 * ks + (mi & 1)) ^ rr) << 4), b00, b01, b10, b11);
-                    ptx::mma_bf16(sacc[0], qa[ks][0], 0u, qa[ks][1], 0u, b00, b01);
-                    ptx::mma_bf16(sacc[1], qa[ks][0], 0u, qa[ks][1], 0u, b10, b11);
+                for (int j = 0; j < 8; ++j) { oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f; }
+                {
+                    const int b = mt.unit / p.kv_heads, g = mt.unit - b * p.kv_heads;
+                    lg = L.logit + ((size_t)b * p.q_heads + (size_t)g * G + min(head, G - 1)) * p.lstride;
                 }
-                // ---------------- online softmax in registers (fp32) -------------------------
-                float s[4] = {sacc[0][0], sacc[0][1], sacc[1][0], sacc[1][1]};
-                const int trow[4] = {blk0 + tk0, blk0 + tk0 + 1, blk0 + tk0 + 8, blk0 + tk0 + 9};
+                if (mt.kind == kEntryTile) {
+                    const uint8_t* qs = qslots + (size_t)stage * kQSlotBytes + (size_t)min(head, G - 1) * kRowB + tk0 * 2;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) s[i] = (trow[i] < nv) ? s[i] * p.scale_log2 : kNegBig;
-                if (dec && mt.seg == 1 && head < G) {
-                    float* lg = L.logit + ((size_t)b * p.q_heads + (size_t)g * G + head) * p.cap + mt.row;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i)
-                        if (trow[i] < nv) lg[trow[i]] = s[i];
-                }
-                float mx = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                const float m_new = fmaxf(m_run, mx);
-                const float sc = fast_exp2(m_run - m_new);
-                float pr[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) pr[i] = fast_exp2(s[i] - m_new);
-                l_run = fmaf(l_run, sc, (pr[0] + pr[1]) + (pr[2] + pr[3]));
-                m_run = m_new;
-                if (sc != 1.0f) {
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) { oacc[j][0] *= sc; oacc[j][1] *= sc; }
-                }
-                // P = hi + lo in bf16: the product with V then carries ~16 mantissa bits of P
-                const uint32_t ahi0 = ptx::pack_bf16x2(pr[0], pr[1]);
-                const uint32_t ahi2 = ptx::pack_bf16x2(pr[2], pr[3]);
-                const uint32_t alo0 = ptx::pack_bf16x2(pr[0] - __uint_as_float(ahi0 << 16),
-                                                       pr[1] - __uint_as_float(ahi0 & 0xffff0000u));
-                const uint32_t alo2 = ptx::pack_bf16x2(pr[2] - __uint_as_float(ahi2 << 16),
-                                                       pr[3] - __uint_as_float(ahi2 & 0xffff0000u));
-                // ---------------- O += P V ------------------------------------------------------
-                const uint32_t vbase = ptx::smem_u32(sV) + (uint32_t)(blk0 + (mi & 1) * 8 + rr) * kRowB;
-#pragma unroll
-                for (int j = 0; j < 16; j += 2) {
-                    uint32_t b0, b1, b2, b3;
-                    ptx::ldmatrix_x4_trans(vbase + (uint32_t)(((j + (mi >> 1)) ^ rr) << 4), b0, b1, b2, b3);
-                    ptx::mma_bf16(oacc[j], ahi0, 0u, ahi2, 0u, b0, b1);
-                    ptx::mma_bf16(oacc[j], alo0, 0u, alo2, 0u, b0, b1);
-                    ptx::mma_bf16(oacc[j + 1], ahi0, 0u, ahi2, 0u, b2, b3);
-                    ptx::mma_bf16(oacc[j + 1], alo0, 0u, alo2, 0u, b2, b3);
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t x0 = *reinterpret_cast<const uint32_t*>(qs + 32 * ks);
+                        const uint32_t x1 = *reinterpret_cast<const uint32_t*>(qs + 32 * ks + 16);
+                        qa[ks][0] = head < G ? x0 : 0u;
+                        qa[ks][1] = head < G ? x1 : 0u;
+                    }
                 }
             }
-            if (wrote) ptx::fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->empty[stage]));
-            if (++stage == nst) { stage = 0; phase ^= 1u; }
-
-            if (mt.last) {
-                // ---------------- item end: merge the four warps, one partial, ticket -----------
+            if (mt.kind == kEntryTile) {
+                const int nv = mt.cnt;
+                bool wrote = false;
+                if (nv > blk0 && nv < blk0 + 16) {
+                    // rows past the valid ones enter the second mma with probability 0: their V
+                    // bytes must be finite, so clear them (stale shared memory may hold anything)
+                    const int nz = (blk0 + 16 - nv) * 16;
+                    for (int idx = lane; idx < nz; idx += 32)
+                        *reinterpret_cast<uint4*>(sV + (size_t)(nv + (idx >> 4)) * kRowB + ((idx & 15) << 4)) =
+                            make_uint4(0u, 0u, 0u, 0u);
+                    wrote = true;
+                    __syncwarp();
+                }
+                if (nv > blk0) {
+                    // ---------------- S = Q K^T: 8 heads (M, padded to 16) x 16 tokens -------------
+                    float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+                    const uint32_t roff = (uint32_t)(blk0 + (mi >> 1) * 8 + rr) * kRowB;
+                    const uint32_t kbase = ptx::smem_u32(sK) + roff;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        uint32_t b00, b01, b10, b11;
+                        ptx::ldmatrix_x4(kbase + (uint32_t)(((2 * ks + (mi & 1)) ^ rr) << 4), b00, b01, b10, b11);
+                        ptx::mma_bf16(sacc[0], qa[ks][0], 0u, qa[ks][1], 0u, b00, b01);
+                        ptx::mma_bf16(sacc[1], qa[ks][0], 0u, qa[ks][1], 0u, b10, b11);
+                    }
+                    // ---------------- online softmax in registers (fp32) -------------------------
+                    float s[4] = {sacc[0][0], sacc[0][1], sacc[1][0], sacc[1][1]};
+                    const int trow[4] = {blk0 + tk0, blk0 + tk0 + 1, blk0 + tk0 + 8, blk0 + tk0 + 9};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) s[i] = (trow[i] < nv) ? s[i] * p.scale_log2 : kNegBig;
+                    if (dec && mt.seg == 1 && head < G) {
+                        float* lr = lg + mt.row;
+                        if (trow[1] < nv) *reinterpret_cast<float2*>(lr + trow[0]) = make_float2(s[0], s[1]);
+                        else if (trow[0] < nv) lr[trow[0]] = s[0];
+                        if (trow[3] < nv) *reinterpret_cast<float2*>(lr + trow[2]) = make_float2(s[2], s[3]);
+                        else if (trow[2] < nv) lr[trow[2]] = s[2];
+                    }
+                    float mx = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                    const float m_new = fmaxf(m_run, mx);
+                    const float sc = fast_exp2(m_run - m_new);
+                    float pr[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) pr[i] = fast_exp2(s[i] - m_new);
+                    l_run = fmaf(l_run, sc, (pr[0] + pr[1]) + (pr[2] + pr[3]));
+                    m_run = m_new;
+                    if (__any_sync(0xffffffffu, sc != 1.0f)) {
+                        // O^T holds heads 2*(lane&3) and +1 in its columns: fetch their factors
+                        const float scA = __shfl_sync(0xffffffffu, sc, (lane & 3) * 8);
+                        const float scB = __shfl_sync(0xffffffffu, sc, (lane & 3) * 8 + 4);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) { oacc[j][0] *= scA; oacc[j][1] *= scB; oacc[j][2] *= scA; oacc[j][3] *= scB; }
+                    }
+                    // P^T as B operand (tokens in K, heads in N).  P = hi + lo in bf16: the
+                    // product with V then carries ~16 mantissa bits of P.
+                    const uint32_t bhi0 = ptx::pack_bf16x2(pr[0], pr[1]);
+                    const uint32_t bhi1 = ptx::pack_bf16x2(pr[2], pr[3]);
+                    const uint32_t blo0 = ptx::pack_bf16x2(pr[0] - __uint_as_float(bhi0 << 16),
+                                                           pr[1] - __uint_as_float(bhi0 & 0xffff0000u));
+                    const uint32_t blo1 = ptx::pack_bf16x2(pr[2] - __uint_as_float(bhi1 << 16),
+                                                           pr[3] - __uint_as_float(bhi1 & 0xffff0000u));
+                    // ---------------- O^T += V^T P^T -------------------------------------------------
+                    const uint32_t vbase = ptx::smem_u32(sV) + roff;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        uint32_t a0, a1, a2, a3;
+                        ptx::ldmatrix_x4_trans(vbase + (uint32_t)(((2 * j + (mi & 1)) ^ rr) << 4), a0, a1, a2, a3);
+                        ptx::mma_bf16(oacc[j], a0, a1, a2, a3, bhi0, bhi1);
+                        ptx::mma_bf16(oacc[j], a0, a1, a2, a3, blo0, blo1);
+                    }
+                }
+                if (wrote) ptx::fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->empty[stage]));
+            } else {
+                // ---------------- item end: hand (m, l, O) to the tail warps ------------------------
                 l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
                 l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-                MergeSmem<GR>& mg = scratch->merge;
-                constexpr int NH = MergeSmem<GR>::NH, HC = MergeSmem<GR>::HC;
-                if ((lane & 3) == 0 && head < GR) { mg.xm[warp][head] = m_run; mg.xl[warp][head] = l_run; }
-                const size_t part = (size_t)mt.item;
+                float* xo = reinterpret_cast<float*>(sK);
+                float* xm = xo + kConsumerWarps * kMaxGroup * kXoStride;
+                float* xl = xm + kConsumerWarps * kMaxGroup;
+                if ((lane & 3) == 0) { xm[warp * kMaxGroup + head] = m_run; xl[warp * kMaxGroup + head] = l_run; }
+                float* oA = xo + (size_t)(warp * kMaxGroup + tk0) * kXoStride + head;   // head tk0, dim lane>>2
+                float* oB = oA + kXoStride;                                              // head tk0 + 1
 #pragma unroll
-                for (int half = 0; half < NH; ++half) {
-                    if (head < GR) {
-#pragma unroll
-                        for (int jj = 0; jj < 16 / NH; ++jj) {
-                            const int j = half * (16 / NH) + jj;
-                            *reinterpret_cast<float2*>(&mg.xo[warp][head][jj * 8 + tk0]) =
-                                make_float2(oacc[j][0], oacc[j][1]);
-                        }
-                    }
-                    bar_sync(1, kConsumers);
-                    for (int idx = tid; idx < G * HC; idx += kConsumers) {
-                        const int row = idx / HC, col = idx - row * HC;
-                        float M = mg.xm[0][row];
-#pragma unroll
-                        for (int w = 1; w < kConsumerWarps; ++w) M = fmaxf(M, mg.xm[w][row]);
-                        float acc = 0.f, ls = 0.f;
-#pragma unroll
-                        for (int w = 0; w < kConsumerWarps; ++w) {
-                            const float wsc = fast_exp2(mg.xm[w][row] - M);
-                            acc = fmaf(mg.xo[w][row][col], wsc, acc);
-                            ls = fmaf(mg.xl[w][row], wsc, ls);
-                        }
-                        L.part_o[(part * G + row) * 128 + half * HC + col] = acc;
-                        if (half == 0 && col == 0) {
-                            L.part_ml[(part * G + row) * 2] = M;
-                            L.part_ml[(part * G + row) * 2 + 1] = ls;
-                        }
-                    }
-                    __threadfence();
-                    bar_sync(1, kConsumers);
+                for (int j = 0; j < 8; ++j) {
+                    oA[16 * j] = oacc[j][0]; oB[16 * j] = oacc[j][1];
+                    oA[16 * j + 8] = oacc[j][2]; oB[16 * j + 8] = oacc[j][3];
                 }
-                if (tid == 0) ctl->last_flag = (atomicAdd(&L.ticket[u], 1) == L.unit_nparts[u] - 1);
-                bar_sync(1, kConsumers);
-                if (ctl->last_flag) {
-                    __threadfence();
-                    unit_tail<kConsumers, 1>(p, u, scratch->tail, tid, kRowB);
-                    bar_sync(1, kConsumers);
+                const int xs = xcount % nst;
+                if (warp == 0 && lane == 0) { ctl->xq[xs].stage = stage; ctl->xq[xs].unit = mt.unit; ctl->xq[xs].item = mt.item; }
+                ptx::fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->xfull[xs]));
+                ++xcount;
+            }
+            if (++stage == nst) { stage = 0; phase ^= 1u; }
+        }
+    } else {
+        // ================================ tail warps ===================================
+        const int tt = tid - kTailTid0;
+        const int n_mine = item_end - item_begin;
+        for (int x = 0; x < n_mine; ++x) {
+            const int xs = x % nst;
+            if (tt == 0) {
+                const bool got = wait_or_abort(ptx::smem_u32(&ctl->xfull[xs]), (uint32_t)((x / nst) & 1), ctl);
+                if (!got && !aborted(ctl)) note_timeout(p, ctl);
+                ctl->wait_ok = got ? 1 : 0;
+            }
+            bar_sync(1, kTailThreads);
+            if (!ctl->wait_ok) break;
+            const ExchangeRef ref = ctl->xq[xs];
+            const int u = ref.unit;
+            const float* xo = reinterpret_cast<const float*>(stages + (size_t)ref.stage * kStageBytes);
+            const float* xm = xo + kConsumerWarps * kMaxGroup * kXoStride;
+            const float* xl = xm + kConsumerWarps * kMaxGroup;
+            const size_t part = (size_t)ref.item;
+            for (int idx = tt; idx < G * 128; idx += kTailThreads) {
+                const int h = idx >> 7, col = idx & 127;
+                float M = xm[h];
+#pragma unroll
+                for (int w = 1; w < kConsumerWarps; ++w) M = fmaxf(M, xm[w * kMaxGroup + h]);
+                float acc = 0.f, ls = 0.f;
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) {
+                    const float wsc = fast_exp2(xm[w * kMaxGroup + h] - M);
+                    acc = fmaf(xo[(size_t)(w * kMaxGroup + h) * kXoStride + col], wsc, acc);
+                    ls = fmaf(xl[w * kMaxGroup + h], wsc, ls);
+                }
+                L.part_o[(part * G + h) * 128 + col] = acc;
+                if (col == 0) {
+                    L.part_ml[(part * G + h) * 2] = M;
+                    L.part_ml[(part * G + h) * 2 + 1] = ls;
                 }
             }
+            __threadfence();
+            ptx::fence_proxy_async();
+            bar_sync(1, kTailThreads);
+            // the borrowed stage goes back to the producer
+            if ((tt & 31) == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->empty[ref.stage]));
+            if (tt == 0) ctl->last_flag = (atomicAdd(&L.ticket[u], 1) == L.unit_nparts[u] - 1);
+            bar_sync(1, kTailThreads);
+            if (ctl->last_flag) {
+                __threadfence();
+                unit_tail<__nv_bfloat16, kTailThreads, 1>(p, u, *tsm, tt);
+            }
+            bar_sync(1, kTailThreads);
         }
     }
-    __syncthreads();
-    if (tid == 0) grid_epilogue(p, gridDim.x);
 }
 
 int g_stages = 3;
@@ -355,22 +404,17 @@ int g_stages = 3;
 }  // namespace
 
 bool mma_supported(int kv_dtype, int head_dim, int group) {
-    return kv_dtype == 0 && head_dim == 128 && group >= 1 && group <= 8;
+    return kv_dtype == 0 && head_dim == 128 && group >= 1 && group <= kMaxGroup;
 }
 
 cudaError_t mma_configure() {
     if (const char* e = std::getenv("MKV_STAGES")) g_stages = max(2, min(kMaxStages, atoi(e)));
-    cudaError_t err = cudaFuncSetAttribute(mma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)smem_bytes<4>(g_stages));
-    if (err != cudaSuccess) return err;
-    return cudaFuncSetAttribute(mma_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)smem_bytes<8>(g_stages));
+    return cudaFuncSetAttribute(mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(g_stages));
 }
 
-cudaError_t launch_mma(const Params& p, int n_ctas, cudaStream_t st) {
-    if (p.L.n_items <= 0) return cudaSuccess;
-    if (p.group <= 4) mma_kernel<4><<<n_ctas, kThreads, smem_bytes<4>(g_stages), st>>>(p, g_stages);
-    else mma_kernel<8><<<n_ctas, kThreads, smem_bytes<8>(g_stages), st>>>(p, g_stages);
+cudaError_t launch_mma(const Params& p, cudaStream_t st) {
+    if (p.L.n_ctas <= 0) return cudaSuccess;
+    mma_kernel<<<p.L.n_ctas, kThreads, smem_bytes(g_stages), st>>>(p, g_stages);
     return cudaGetLastError();
 }
 

@@ -1,18 +1,25 @@
 // Tail of one unit (sequence b, KV head g), run by the thread group that delivered the
 // unit's last partial.  In order:
+//   0. the fresh token of the step (Algorithm 1, append): its logit q_h . k_new / sqrt(d)
+//      for the G heads; it takes part in the softmax as one more partial
+//      (m = its logit, l = 1, O = v_new).
 //   1. cross-split log-sum-exp combine: global max M_h and sum L_h per query head,
-//      out_h = sum_p O_p 2^(m_p - M_h) / L_h                      (Eq. 2)
-//   2. normalised probability of every decode token, including the fresh one, from the
-//      stored raw logits: p = 2^(s - M_h) / L_h; mean over the G heads  (Eq. 4)
-//   3. I_i <- beta * I_i + abar_i, the fresh token starting from 0    (Eq. 5, Eq. 6)
+//      out_h = (sum_p O_p 2^(m_p - M_h) + v_new 2^(s_new - M_h)) / L_h        (Eq. 2)
+//   2. normalised probability of every decode token from the stored raw logits:
+//      p = 2^(s - M_h) / L_h; mean over the G heads                           (Eq. 4)
+//   3. I_i <- beta * I_i + abar_i; the fresh token starts from 0              (Eq. 5, 6)
 //   4. overflow k = max(0, n - budget) (Eq. 7); the k smallest 64-bit keys
 //      (fp32 score bits, position id) are the evicted set (Eq. 8).  Scores are
 //      non-negative so their bit patterns order like the values: selection is integer
 //      work on exactly the scores that are stored.  k = 1: arg-min reduction.
 //      k > 1: 8-pass byte-wise radix select of the k-th key.
-//   5. compaction (Eq. 9): survivors stored beyond the new count move into the holes
-//      (K row, V row, score, position id); slot order changes, which is harmless because
-//      softmax and sum(p v) do not depend on the order and ties are broken by position id.
+//   5. append + compaction (Eq. 9).  k = 0: the fresh row goes to slot n_old.  k = 1: the
+//      fresh row goes straight into the evicted slot (nothing is written when the fresh
+//      token itself is the one evicted), which leaves the pool exactly as "append at the
+//      end, then move the last row into the hole" would.  k > 1: append, then survivors
+//      stored beyond the new count move into the holes (K row, V row, score, position id).
+//      Slot order changes, which is harmless: softmax and sum(p v) do not depend on the
+//      order and ties are broken by position id.
 // NT threads take part (a multiple of 32); they synchronise on named barrier BAR only,
 // so a subset of a CTA can run the tail while other warps keep streaming.
 #pragma once
@@ -24,6 +31,8 @@ template <int NT>
 struct TailSmem {
     float M[kMaxGroup];
     float invL[kMaxGroup];
+    float snew[kMaxGroup];   // logit of the fresh token (log2 units)
+    float wnew[kMaxGroup];   // 2^(snew - M)
     float w[kMaxParts][kMaxGroup];
     unsigned long long red_key[NT / 32];
     int red_slot[NT / 32];
@@ -40,21 +49,47 @@ __device__ inline void copy_row_swizzled(uint8_t* pool, size_t unit_base, int ro
     for (int c = lane; c < chunks; c += 32) d[c ^ (dst & 7)] = __ldcg(&s[c ^ (src & 7)]);
 }
 
-template <int NT, int BAR>
-__device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid, int rowb) {
+// plain row (k_new / v_new of the unit) -> pool slot `dst`, chunk-permuted
+__device__ inline void store_row_swizzled(uint8_t* pool, size_t unit_base, int rowb, const void* src_row, int dst,
+                                          int lane) {
+    const int chunks = rowb >> 4;
+    const uint4* s = reinterpret_cast<const uint4*>(src_row);
+    uint4* d = reinterpret_cast<uint4*>(pool + unit_base + (size_t)dst * rowb);
+    for (int c = lane; c < chunks; c += 32) d[c ^ (dst & 7)] = __ldg(&s[c]);
+}
+
+template <typename T, int NT, int BAR>
+__device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid) {
     const LayerDev& L = p.L;
     const int G = p.group, D = p.head_dim, cap = p.cap;
+    const int rowb = D * (int)sizeof(T);
     const int b = u / p.kv_heads, g = u - b * p.kv_heads;
     const int P = L.unit_nparts[u], part0 = L.unit_part0[u];
-    const int n_old = L.n_dec[u];
     const bool dec = (p.mode == kModeDecode);
-    const int n = dec ? min(n_old + 1, cap) : n_old;
+    const int n_old = min(L.n_dec[u], dec ? cap - 1 : cap);
+    const int n = dec ? n_old + 1 : n_old;
+    const int t = L.unit_step[u];     // read before the first barrier: thread 0 advances it below
     const int lane = tid & 31, warp = tid >> 5;
     constexpr int NW = NT / 32;
+    const T* qrow = reinterpret_cast<const T*>(p.q) + ((size_t)b * p.q_heads + (size_t)g * G) * D;
+    const T* knew = reinterpret_cast<const T*>(p.k_new) + (size_t)u * D;
+    const T* vnew = reinterpret_cast<const T*>(p.v_new) + (size_t)u * D;
 
-    // ---- 1. combine -------------------------------------------------------------------
+    // ---- 0. logit of the fresh token ------------------------------------------------------
+    if (dec) {
+        for (int h = warp; h < G; h += NW) {
+            float a = 0.f;
+            for (int e = lane; e < D; e += 32) a = fmaf(to_f32(qrow[(size_t)h * D + e]), to_f32(knew[e]), a);
+#pragma unroll
+            for (int off = 16; off; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
+            if (lane == 0) sm.snew[h] = a * p.scale_log2;
+        }
+        bar_sync(BAR, NT);
+    }
+
+    // ---- 1. combine -----------------------------------------------------------------------
     if (tid < G) {
-        float M = kNegBig;
+        float M = dec ? sm.snew[tid] : kNegBig;
         for (int q = 0; q < P; ++q) M = fmaxf(M, __ldcg(&L.part_ml[((size_t)(part0 + q) * G + tid) * 2]));
         float Lsum = 0.f;
         for (int q = 0; q < P; ++q) {
@@ -63,6 +98,9 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid, int
             sm.w[q][tid] = w;
             Lsum += ml.y * w;
         }
+        float wn = 0.f;
+        if (dec) { wn = fast_exp2(sm.snew[tid] - M); Lsum += wn; }
+        sm.wnew[tid] = wn;
         sm.M[tid] = M;
         sm.invL[tid] = Lsum > 0.f ? 1.0f / Lsum : 0.f;
     }
@@ -71,7 +109,7 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid, int
         const size_t obase = ((size_t)b * p.q_heads + (size_t)g * G) * D;
         for (int idx = tid; idx < G * D; idx += NT) {
             const int h = idx / D;
-            float acc = 0.f;
+            float acc = dec ? to_f32(vnew[idx - h * D]) * sm.wnew[h] : 0.f;
             for (int q = 0; q < P; ++q)
                 acc = fmaf(__ldcg(&L.part_o[(size_t)(part0 + q) * G * D + idx]), sm.w[q][h], acc);
             acc *= sm.invL[h];
@@ -85,37 +123,47 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid, int
     }
 
     // ---- 2./3. probabilities, head mean, momentum update ---------------------------------
-    const int t = L.step[0];
     const int k = max(0, n - p.budget);
     const float inv_g = 1.0f / (float)G;
     float* score = L.score + (size_t)u * cap;
     int32_t* pos = L.pos + (size_t)u * cap;
     unsigned long long* keys = L.keys + (size_t)u * cap;
-    const float* lg = L.logit + ((size_t)b * p.q_heads + (size_t)g * G) * cap;
+    const float* lg = L.logit + ((size_t)b * p.q_heads + (size_t)g * G) * p.lstride;
+    float ab_new = 0.f;
+    for (int h = 0; h < G; ++h) ab_new += sm.wnew[h] * sm.invL[h];
+    ab_new *= inv_g;                                  // Eq. 6: I_fresh = alpha * 0 + abar_fresh
+    const unsigned long long key_new = ((unsigned long long)__float_as_uint(ab_new) << 32) | (unsigned)t;
     unsigned long long best_key = ~0ull;
     int best_slot = -1;
-    for (int i = tid; i < n; i += NT) {
+    for (int i = tid; i < n_old; i += NT) {
         float s = 0.f;
-        for (int h = 0; h < G; ++h) s += fast_exp2(__ldcg(&lg[(size_t)h * cap + i]) - sm.M[h]) * sm.invL[h];
+        for (int h = 0; h < G; ++h) s += fast_exp2(__ldcg(&lg[(size_t)h * p.lstride + i]) - sm.M[h]) * sm.invL[h];
         const float ab = s * inv_g;
-        const bool fresh = (i == n - 1);
-        const float old = fresh ? 0.f : score[i];
-        const float nw = fmaf(p.beta, old, ab);
-        const int ps = fresh ? t : pos[i];
+        const float nw = fmaf(p.beta, score[i], ab);
         score[i] = nw;
-        if (fresh) pos[i] = t;
         if (L.abar) L.abar[(size_t)u * cap + i] = ab;
-        const unsigned long long key = ((unsigned long long)__float_as_uint(nw) << 32) | (unsigned)ps;
+        const unsigned long long key = ((unsigned long long)__float_as_uint(nw) << 32) | (unsigned)pos[i];
         if (k > 1) keys[i] = key;
         if (key < best_key) { best_key = key; best_slot = i; }
     }
-    if (tid == 0) { L.n_prev[u] = n; L.ev_k[u] = k; L.n_dec[u] = n - k; }
-    if (k == 0) {
-        if (tid == 0) L.ticket[u] = 0;
-        return;
+    if (tid == NT - 1) {                              // the fresh token sits (virtually) in slot n_old
+        if (key_new < best_key) { best_key = key_new; best_slot = n_old; }
+        if (L.abar) L.abar[(size_t)u * cap + n_old] = ab_new;
     }
+    if (tid == 0) { L.n_prev[u] = n; L.ev_k[u] = k; L.n_dec[u] = n - k; L.unit_step[u] = t + 1; }
 
     const size_t ubase = (size_t)u * cap * rowb;
+    if (k != 1) {
+        // ---- 5 (k = 0, and first half of k > 1): append at the end ----------------------
+        if (warp == 0) store_row_swizzled(L.Kd, ubase, rowb, knew, n_old, lane);
+        if (warp == (NW > 1 ? 1 : 0)) store_row_swizzled(L.Vd, ubase, rowb, vnew, n_old, lane);
+        if (tid == NT - 1) { score[n_old] = ab_new; pos[n_old] = t; keys[n_old] = key_new; }
+        if (k == 0) {
+            if (tid == 0) L.ticket[u] = 0;
+            return;
+        }
+    }
+
     if (k == 1) {
         // ---- 4a. arg-min over (score bits, position id) ------------------------------
         for (int off = 16; off; off >>= 1) {
@@ -124,26 +172,27 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid, int
             if (ok < best_key) { best_key = ok; best_slot = os; }
         }
         if (lane == 0) { sm.red_key[warp] = best_key; sm.red_slot[warp] = best_slot; }
-        bar_sync(BAR, NT);   // also orders every score/pos write before the move below
+        bar_sync(BAR, NT);   // also orders every score write before the stores below
         unsigned long long kk = sm.red_key[0];
         int e = sm.red_slot[0];
         for (int w2 = 1; w2 < NW; ++w2)
             if (sm.red_key[w2] < kk) { kk = sm.red_key[w2]; e = sm.red_slot[w2]; }
-        // ---- 5a. the fresh slot n-1 is the only possible mover ------------------------
         if (tid == 0) {
             L.ev_pos[(size_t)u * cap] = (int32_t)(unsigned)(kk & 0xffffffffu);
             L.ev_score[(size_t)u * cap] = __uint_as_float((unsigned)(kk >> 32));
         }
-        if (e != n - 1) {
-            if (warp == 0) copy_row_swizzled(L.Kd, ubase, rowb, n - 1, e, lane);
-            if (warp == (NW > 1 ? 1 : 0)) copy_row_swizzled(L.Vd, ubase, rowb, n - 1, e, lane);
-            if (tid == NT - 1) { score[e] = score[n - 1]; pos[e] = pos[n - 1]; }
+        // ---- 5a. the fresh row lands in the hole -----------------------------------------
+        if (e != n_old) {
+            if (warp == 0) store_row_swizzled(L.Kd, ubase, rowb, knew, e, lane);
+            if (warp == (NW > 1 ? 1 : 0)) store_row_swizzled(L.Vd, ubase, rowb, vnew, e, lane);
+            if (tid == NT - 1) { score[e] = ab_new; pos[e] = t; }
         }
         if (tid == 0) L.ticket[u] = 0;
         return;
     }
 
     // ---- 4b. radix select of the k-th smallest key (keys are distinct) ----------------
+    bar_sync(BAR, NT);       // keys, scores and the appended row are in place
     unsigned long long prefix = 0ull, mask = 0ull;
     int want = k - 1;
     for (int pass = 7; pass >= 0; --pass) {
