@@ -61,8 +61,8 @@ bool make_layout(int layers, int batch, int q_heads, int kv_heads, int head_dim,
     L.lo.Vp = take(U * max_prefill * L.rowb);
     L.lo.Kd = take(U * C * L.rowb);
     L.lo.Vd = take(U * C * L.rowb);
-    L.lo.score = take(U * C * 4);
-    L.lo.pos = take(U * C * 4);
+    L.lo.score = take(U * L.lstride * 4);
+    L.lo.pos = take(U * L.lstride * 4);
     L.lo.n_dec = take(U * 4);
     L.lo.logit = take((size_t)batch * q_heads * L.lstride * 4);
     L.lo.abar = take(U * C * 4);
@@ -454,8 +454,8 @@ mkv_status mkv_get_decode_state(mkv_ctx* c, int layer, int b, int g, int32_t* n,
     const int u = b * c->kv_heads + g;
     MKV_D2H(n, d.n_dec + u, 4);
     if ((pos || score) && *n > cap) return MKV_ERR_CAPACITY;
-    if (pos) MKV_D2H(pos, d.pos + (size_t)u * c->lay.cap, (size_t)*n * 4);
-    if (score) MKV_D2H(score, d.score + (size_t)u * c->lay.cap, (size_t)*n * 4);
+    if (pos) MKV_D2H(pos, d.pos + (size_t)u * c->lay.lstride, (size_t)*n * 4);
+    if (score) MKV_D2H(score, d.score + (size_t)u * c->lay.lstride, (size_t)*n * 4);
     return MKV_OK;
 }
 

@@ -39,7 +39,7 @@ namespace mkv {
 
 constexpr int kTileRows = 64;       // rows of one tile of the work decomposition
 constexpr int kMaxGroup = 8;        // G = q_heads / kv_heads the kernels are built for
-constexpr int kMaxParts = 128;      // partials per unit (CTA ranges grow to keep this)
+constexpr int kMaxParts = 64;       // partials per unit (CTA ranges grow to keep this)
 constexpr int kMaxCtas = 2048;      // persistent grid upper bound (sizes the partial scratch)
 constexpr float kNegBig = -1.0e30f; // finite stand-in for -inf in running maxima
 

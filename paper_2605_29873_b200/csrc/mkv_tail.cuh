@@ -33,7 +33,8 @@ struct TailSmem {
     float invL[kMaxGroup];
     float snew[kMaxGroup];   // logit of the fresh token (log2 units)
     float wnew[kMaxGroup];   // 2^(snew - M)
-    float w[kMaxParts][kMaxGroup];
+    float w[kMaxParts][kMaxGroup];    // running max of a partial, then its weight 2^(m - M)
+    float pl[kMaxParts][kMaxGroup];   // running sum of a partial
     unsigned long long red_key[NT / 32];
     int red_slot[NT / 32];
     int hist[256];
@@ -61,7 +62,7 @@ __device__ inline void store_row_swizzled(uint8_t* pool, size_t unit_base, int r
 template <typename T, int NT, int BAR>
 __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid) {
     const LayerDev& L = p.L;
-    const int G = p.group, D = p.head_dim, cap = p.cap;
+    const int G = p.group, D = p.head_dim, cap = p.cap, ls = p.lstride;
     const int rowb = D * (int)sizeof(T);
     const int b = u / p.kv_heads, g = u - b * p.kv_heads;
     const int P = L.unit_nparts[u], part0 = L.unit_part0[u];
@@ -74,7 +75,34 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid) {
     const T* qrow = reinterpret_cast<const T*>(p.q) + ((size_t)b * p.q_heads + (size_t)g * G) * D;
     const T* knew = reinterpret_cast<const T*>(p.k_new) + (size_t)u * D;
     const T* vnew = reinterpret_cast<const T*>(p.v_new) + (size_t)u * D;
+    float* score = L.score + (size_t)u * ls;
+    int32_t* pos = L.pos + (size_t)u * ls;
+    const float* lg = L.logit + ((size_t)b * p.q_heads + (size_t)g * G) * ls;
 
+    // Everything below is latency: a handful of dependent trips to L2.  So every load that
+    // does not need the softmax statistics is issued first, in one batch: the partials'
+    // (m, l), the fresh token's dot products, and this thread's first four tokens' logits,
+    // scores and position ids (as 16-byte vectors).
+    struct Tok { float4 lgv[kMaxGroup]; float4 sc; int4 ps; };
+    auto load_tok = [&](int i0, Tok& r) {
+        if (i0 < n_old) {
+#pragma unroll
+            for (int h = 0; h < kMaxGroup; ++h)
+                if (h < G) r.lgv[h] = __ldcg(reinterpret_cast<const float4*>(lg + (size_t)h * ls + i0));
+            r.sc = *reinterpret_cast<const float4*>(score + i0);
+            r.ps = *reinterpret_cast<const int4*>(pos + i0);
+        }
+    };
+    Tok tk;
+    if (dec) load_tok(4 * tid, tk);
+    for (int e0 = 0; e0 < P * kMaxGroup; e0 += NT) {
+        const int e = e0 + tid, q = e / kMaxGroup, h = e - q * kMaxGroup;
+        if (q < P && h < G) {
+            const float2 ml = __ldcg(reinterpret_cast<const float2*>(&L.part_ml[((size_t)(part0 + q) * G + h) * 2]));
+            sm.w[q][h] = ml.x;
+            sm.pl[q][h] = ml.y;
+        }
+    }
     // ---- 0. logit of the fresh token ------------------------------------------------------
     if (dec) {
         for (int h = warp; h < G; h += NW) {
@@ -84,19 +112,18 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid) {
             for (int off = 16; off; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
             if (lane == 0) sm.snew[h] = a * p.scale_log2;
         }
-        bar_sync(BAR, NT);
     }
+    bar_sync(BAR, NT);
 
     // ---- 1. combine -----------------------------------------------------------------------
     if (tid < G) {
         float M = dec ? sm.snew[tid] : kNegBig;
-        for (int q = 0; q < P; ++q) M = fmaxf(M, __ldcg(&L.part_ml[((size_t)(part0 + q) * G + tid) * 2]));
+        for (int q = 0; q < P; ++q) M = fmaxf(M, sm.w[q][tid]);
         float Lsum = 0.f;
         for (int q = 0; q < P; ++q) {
-            const float2 ml = __ldcg(reinterpret_cast<const float2*>(&L.part_ml[((size_t)(part0 + q) * G + tid) * 2]));
-            const float w = fast_exp2(ml.x - M);
+            const float w = fast_exp2(sm.w[q][tid] - M);
             sm.w[q][tid] = w;
-            Lsum += ml.y * w;
+            Lsum = fmaf(sm.pl[q][tid], w, Lsum);
         }
         float wn = 0.f;
         if (dec) { wn = fast_exp2(sm.snew[tid] - M); Lsum += wn; }
@@ -107,11 +134,19 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid) {
     bar_sync(BAR, NT);
     {
         const size_t obase = ((size_t)b * p.q_heads + (size_t)g * G) * D;
+        const float* po = L.part_o + (size_t)part0 * G * D;
+        const size_t pstride = (size_t)G * D;
         for (int idx = tid; idx < G * D; idx += NT) {
             const int h = idx / D;
             float acc = dec ? to_f32(vnew[idx - h * D]) * sm.wnew[h] : 0.f;
-            for (int q = 0; q < P; ++q)
-                acc = fmaf(__ldcg(&L.part_o[(size_t)(part0 + q) * G * D + idx]), sm.w[q][h], acc);
+            int q = 0;
+            for (; q + 4 <= P; q += 4) {
+                const float v0 = __ldcg(po + (size_t)q * pstride + idx), v1 = __ldcg(po + (size_t)(q + 1) * pstride + idx);
+                const float v2 = __ldcg(po + (size_t)(q + 2) * pstride + idx), v3 = __ldcg(po + (size_t)(q + 3) * pstride + idx);
+                acc = fmaf(v0, sm.w[q][h], acc); acc = fmaf(v1, sm.w[q + 1][h], acc);
+                acc = fmaf(v2, sm.w[q + 2][h], acc); acc = fmaf(v3, sm.w[q + 3][h], acc);
+            }
+            for (; q < P; ++q) acc = fmaf(__ldcg(po + (size_t)q * pstride + idx), sm.w[q][h], acc);
             acc *= sm.invL[h];
             if (p.out_f32) reinterpret_cast<float*>(p.out)[obase + idx] = acc;
             else reinterpret_cast<__nv_bfloat16*>(p.out)[obase + idx] = __float2bfloat16_rn(acc);
@@ -125,26 +160,54 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid) {
     // ---- 2./3. probabilities, head mean, momentum update ---------------------------------
     const int k = max(0, n - p.budget);
     const float inv_g = 1.0f / (float)G;
-    float* score = L.score + (size_t)u * cap;
-    int32_t* pos = L.pos + (size_t)u * cap;
     unsigned long long* keys = L.keys + (size_t)u * cap;
-    const float* lg = L.logit + ((size_t)b * p.q_heads + (size_t)g * G) * p.lstride;
     float ab_new = 0.f;
     for (int h = 0; h < G; ++h) ab_new += sm.wnew[h] * sm.invL[h];
     ab_new *= inv_g;                                  // Eq. 6: I_fresh = alpha * 0 + abar_fresh
     const unsigned long long key_new = ((unsigned long long)__float_as_uint(ab_new) << 32) | (unsigned)t;
     unsigned long long best_key = ~0ull;
     int best_slot = -1;
-    for (int i = tid; i < n_old; i += NT) {
-        float s = 0.f;
-        for (int h = 0; h < G; ++h) s += fast_exp2(__ldcg(&lg[(size_t)h * p.lstride + i]) - sm.M[h]) * sm.invL[h];
-        const float ab = s * inv_g;
-        const float nw = fmaf(p.beta, score[i], ab);
-        score[i] = nw;
-        if (L.abar) L.abar[(size_t)u * cap + i] = ab;
-        const unsigned long long key = ((unsigned long long)__float_as_uint(nw) << 32) | (unsigned)pos[i];
-        if (k > 1) keys[i] = key;
-        if (key < best_key) { best_key = key; best_slot = i; }
+    float Mh[kMaxGroup], iLh[kMaxGroup];
+#pragma unroll
+    for (int h = 0; h < kMaxGroup; ++h) { Mh[h] = h < G ? sm.M[h] : 0.f; iLh[h] = h < G ? sm.invL[h] : 0.f; }
+    for (int base = 0; base < n_old; base += 4 * NT) {
+        const int i0 = base + 4 * tid;
+        if (base > 0) load_tok(i0, tk);
+        if (i0 < n_old) {
+            float ab[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int h = 0; h < kMaxGroup; ++h) {
+                if (h < G) {
+                    ab[0] = fmaf(fast_exp2(tk.lgv[h].x - Mh[h]), iLh[h], ab[0]);
+                    ab[1] = fmaf(fast_exp2(tk.lgv[h].y - Mh[h]), iLh[h], ab[1]);
+                    ab[2] = fmaf(fast_exp2(tk.lgv[h].z - Mh[h]), iLh[h], ab[2]);
+                    ab[3] = fmaf(fast_exp2(tk.lgv[h].w - Mh[h]), iLh[h], ab[3]);
+                }
+            }
+            const float old[4] = {tk.sc.x, tk.sc.y, tk.sc.z, tk.sc.w};
+            const int ps[4] = {tk.ps.x, tk.ps.y, tk.ps.z, tk.ps.w};
+            float nw[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                ab[j] *= inv_g;
+                nw[j] = fmaf(p.beta, old[j], ab[j]);
+            }
+            if (i0 + 4 <= n_old) {
+                *reinterpret_cast<float4*>(score + i0) = make_float4(nw[0], nw[1], nw[2], nw[3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) if (i0 + j < n_old) score[i0 + j] = nw[j];
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (i0 + j < n_old) {
+                    if (L.abar) L.abar[(size_t)u * cap + i0 + j] = ab[j];
+                    const unsigned long long key = ((unsigned long long)__float_as_uint(nw[j]) << 32) | (unsigned)ps[j];
+                    if (k > 1) keys[i0 + j] = key;
+                    if (key < best_key) { best_key = key; best_slot = i0 + j; }
+                }
+            }
+        }
     }
     if (tid == NT - 1) {                              // the fresh token sits (virtually) in slot n_old
         if (key_new < best_key) { best_key = key_new; best_slot = n_old; }
