@@ -102,7 +102,7 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def time_oracle(w, lens, n_units, steps, warmup, time_cap_s):
+def time_oracle(w, lens, n_units, steps, warmup, time_cap_s, min_time_s=0.0):
     """Times the fp64 oracle, as it stands, on a bounded sample of the workload: the first
     `n_units` (sequence, KV head) units, each with its G query heads, from the start of
     generation (empty decode pool), one host thread per unit up to the core count.  Only the
@@ -133,7 +133,9 @@ def time_oracle(w, lens, n_units, steps, warmup, time_cap_s):
     chunk = 128
     total = warmup + steps
     wall0 = time.perf_counter()
-    while t_idx < total:
+    while t_idx < total or elapsed < min_time_s:
+        if t_idx >= total:
+            total += chunk          # keep stepping until the sample holds min_time_s of oracle work
         nb = min(chunk, total - t_idx)
         data = {b: streams[b].next(nb) for b in seq_ids}
         for i in range(nb):
@@ -152,6 +154,10 @@ def time_oracle(w, lens, n_units, steps, warmup, time_cap_s):
                 done["warm"] += 1
             t_idx += 1
             if time.perf_counter() - wall0 > time_cap_s and done["timed"] >= 3:
+                t_idx = total
+                min_time_s = 0.0
+                break
+            if t_idx >= warmup + steps and elapsed >= min_time_s:
                 t_idx = total
                 break
     pool.shutdown()
@@ -355,7 +361,7 @@ def main():
                            "ms_per_step": ms_e2e_max, "sync": "stream synchronised after every step"}
         if not args.no_cpu_baseline and world == 1:
             n_units = min(len(os.sched_getaffinity(0)), B * Hkv)
-            v, threads, sample, _ = time_oracle(w, lens, n_units, steps=48, warmup=2, time_cap_s=25.0)
+            v, threads, sample, _ = time_oracle(w, lens, n_units, steps=48, warmup=2, time_cap_s=40.0, min_time_s=12.0)
             line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": sample}
         print(json.dumps(line), flush=True)
     if world > 1:
