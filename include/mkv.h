@@ -166,6 +166,38 @@ mkv_status mkv_reset(mkv_ctx* ctx);
 /* Synchronise `stream`, then return the sticky device status (MKV_OK if clean). */
 mkv_status mkv_status_sync(mkv_ctx* ctx, void* stream);
 
+/*
+ * Plain decode attention (softmax(q K^T / sqrt(d)) V) for callers that cannot allocate
+ * device memory.  The paper has no counterpart of this call: it exists for hosts that are
+ * handed input and output buffers only -- code running after a serving process has given
+ * all device memory to its own pool, plug-ins without access to an allocator, processes
+ * where allocation is forbidden once serving has begun.  It needs no context and no
+ * workspace.  What its CTAs exchange (split-KV partials, tickets) lives in a fixed array
+ * inside the library image, about 4.3 MB that every GPU loading the library holds until
+ * the process exits; that array bounds the problem size:
+ *     batch * kv_heads                         <= MKV_NOALLOC_MAX_UNITS
+ *     batch * q_heads * ceil(n_tokens / 256)   <= MKV_NOALLOC_MAX_PART_ROWS
+ *     n_tokens                                 <= 16384
+ * Larger problems are refused with MKV_ERR_CAPACITY.
+ *   q    device pointer [batch][q_heads][head_dim], kv_dtype
+ *   K,V  device pointers [batch][kv_heads][kv_rows][head_dim], kv_dtype, plain row order;
+ *        every sequence attends rows [0, n_tokens)
+ *   out  device pointer [batch][q_heads][head_dim], out_dtype
+ *   head_dim 64 or 128, q_heads / kv_heads <= 8, device = CUDA ordinal of the buffers
+ * Asynchronous on `stream`.  The call allocates nothing and frees nothing.  The first call
+ * on a device looks up the device address of the built-in array; make that first call
+ * before starting any stream capture.  All calls share the one array, which keeps the
+ * previous call's contents (tickets are cleared on `stream` at the start of every call):
+ * calls whose kernels may overlap on the GPU -- different streams, several host threads --
+ * race on it and must be ordered by the caller.
+ * Errors: INVALID_ARG, UNSUPPORTED (head_dim, group size), CAPACITY, CUDA.
+ */
+#define MKV_NOALLOC_MAX_UNITS 2048
+#define MKV_NOALLOC_MAX_PART_ROWS 8192
+mkv_status mkv_attend_noalloc(const void* q, const void* K, const void* V, void* out, int batch,
+                              int q_heads, int kv_heads, int head_dim, int n_tokens, int kv_rows,
+                              int kv_dtype, int out_dtype, int device, void* stream);
+
 /* Number of kernels this context has launched so far (host counter). */
 int64_t mkv_launch_count(const mkv_ctx* ctx);
 

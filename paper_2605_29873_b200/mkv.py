@@ -21,7 +21,7 @@ EXPORTED_SYMBOLS = [
     "mkv_workspace_bytes", "mkv_kv_bytes_per_token", "mkv_create", "mkv_destroy", "mkv_prefill",
     "mkv_decode_step", "mkv_decode_step_host", "mkv_attend_only", "mkv_set_budget", "mkv_reset",
     "mkv_status_sync", "mkv_launch_count", "mkv_get_decode_state", "mkv_get_last_evicted",
-    "mkv_get_last_probs", "mkv_read_kv", "mkv_get_step", "mkv_status_string",
+    "mkv_get_last_probs", "mkv_read_kv", "mkv_get_step", "mkv_status_string", "mkv_attend_noalloc",
 ]
 
 
@@ -66,6 +66,7 @@ def load_library(path: str | None = None):
     L.mkv_get_last_probs.argtypes = [vp, C.c_int, C.c_int, C.c_int, i32p, f32p, C.c_int]
     L.mkv_read_kv.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, i32p, vp, vp, C.c_int]
     L.mkv_get_step.argtypes = [vp, C.c_int, C.POINTER(C.c_int64)]
+    L.mkv_attend_noalloc.argtypes = [vp, vp, vp, vp] + [C.c_int] * 9 + [vp]
     L.mkv_status_string.restype = C.c_char_p
     L.mkv_status_string.argtypes = [C.c_int]
     if path is None:
@@ -85,6 +86,25 @@ def workspace_bytes(layers, batch, q_heads, kv_heads, head_dim, budget, max_pref
 
 def kv_bytes_per_token(layers, kv_heads, head_dim, kv_dtype=MKV_BF16) -> int:
     return int(load_library().mkv_kv_bytes_per_token(layers, kv_heads, head_dim, kv_dtype))
+
+
+def attend_noalloc(q, K, V, out, n_tokens, stream=None):
+    """Plain decode attention without context or workspace (``mkv_attend_noalloc``): for
+    callers that may not allocate device memory.  q [B,Hq,d], K/V [B,Hkv,rows,d], out
+    [B,Hq,d] are device tensors; every sequence attends rows [0, n_tokens).  Calls share a
+    scratch array built into the library, so calls on different streams must not overlap."""
+    import torch
+    B, Hq, d = q.shape
+    Hkv, rows = K.shape[1], K.shape[2]
+    assert q.is_contiguous() and K.is_contiguous() and V.is_contiguous() and out.is_contiguous()
+    assert tuple(K.shape) == (B, Hkv, rows, d) == tuple(V.shape) and tuple(out.shape) == (B, Hq, d)
+    assert q.dtype == K.dtype == V.dtype
+    kv = MKV_BF16 if q.dtype == torch.bfloat16 else MKV_F32
+    od = MKV_BF16 if out.dtype == torch.bfloat16 else MKV_F32
+    st = stream if stream is not None else torch.cuda.current_stream(q.device)
+    _check(load_library().mkv_attend_noalloc(_ptr(q), _ptr(K), _ptr(V), _ptr(out), B, Hq, Hkv, d, int(n_tokens),
+                                             rows, kv, od, q.device.index or 0, C.c_void_p(st.cuda_stream)),
+           "mkv_attend_noalloc")
 
 
 def _check(code, where):
