@@ -114,6 +114,24 @@ __device__ inline void bar_sync(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
+// Optional per-CTA timestamps (diagnostic builds only: compile with -DMKV_TRACE).  Slot i of
+// CTA c is g_trace[c * 16 + i]; mkv_debug_trace() copies the array to the host.
+#ifdef MKV_TRACE
+extern __device__ unsigned long long g_trace[kMaxCtas * 16];
+__device__ inline unsigned long long trace_now() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define MKV_TR(i) (mkv::g_trace[blockIdx.x * 16 + (i)] = mkv::trace_now())
+#define MKV_TR_ADD(i, v) (mkv::g_trace[blockIdx.x * 16 + (i)] += (v))
+#define MKV_TR_SET(i, v) (mkv::g_trace[blockIdx.x * 16 + (i)] = (v))
+#else
+#define MKV_TR(i) ((void)0)
+#define MKV_TR_ADD(i, v) ((void)0)
+#define MKV_TR_SET(i, v) ((void)0)
+#endif
+
 // Tile `t` of a unit's tile sequence -> (segment, first row, valid rows).  Prefill tiles
 // come first; decode tiles cover the pool's rows [0, n_old).
 struct TileRef { int seg, row, cnt; };

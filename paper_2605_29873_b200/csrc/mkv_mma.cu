@@ -9,8 +9,9 @@
 //     non-tensor TMA form, no multicast) of K and V tiles, 16 KB each, into a ring of
 //     shared-memory stages; completion is signalled on an mbarrier (complete_tx).  The
 //     cache rows are already chunk-permuted in HBM, so a straight copy lands a layout that
-//     ldmatrix reads without bank conflicts.  The first tile of an item also brings the
-//     unit's G query rows.  The producer runs ahead across item boundaries.
+//     ldmatrix reads without bank conflicts.  At the start of an item it also copies the
+//     unit's G query rows into one of two small query slots.  The producer runs ahead
+//     across item boundaries.
 //   * four CONSUMER warps each own 16 rows of a tile and never synchronise with one
 //     another.  S = Q K^T uses mma.sync m16n8k16 (bf16 in, fp32 accumulate) with the G
 //     query heads in the M dimension; its accumulator fragment is, register for register,
@@ -38,12 +39,17 @@
 #include "mkv_tail.cuh"
 
 namespace mkv {
+#ifdef MKV_TRACE
+__device__ unsigned long long g_trace[kMaxCtas * 16];
+#endif
 namespace {
 
 constexpr int kRowB = 256;                                // 128 bf16
 constexpr int kTileBytes = kTileRows * kRowB;             // 16 KB (K or V)
 constexpr int kStageBytes = 2 * kTileBytes;               // K then V
-constexpr int kQSlotBytes = kMaxGroup * kRowB;            // query rows of one unit
+constexpr int kQRowB = kRowB + 16;                         // padded query row: the heads fall into different banks
+constexpr int kQSlotBytes = kMaxGroup * kQRowB;           // query rows of one unit
+constexpr int kQSlots = 2;
 constexpr int kConsumerWarps = 4;
 constexpr int kTailWarps = 4;
 constexpr int kConsumers = kConsumerWarps * 32;
@@ -73,6 +79,8 @@ struct Control {
     unsigned long long full[kMaxStages];
     unsigned long long empty[kMaxStages];
     unsigned long long xfull[kMaxStages];
+    unsigned long long qfull[kQSlots];
+    unsigned long long qempty[kQSlots];
     StageMeta meta[kMaxStages];
     ExchangeRef xq[kMaxStages];
     int abort_flag;
@@ -81,7 +89,7 @@ struct Control {
 };
 
 constexpr size_t smem_bytes(int nst) {
-    return (size_t)nst * (kStageBytes + kQSlotBytes) + sizeof(TailSmem<kTailThreads>) + sizeof(Control) + 64;
+    return (size_t)nst * kStageBytes + kQSlots * kQSlotBytes + sizeof(TailSmem<kTailThreads>) + sizeof(Control) + 64;
 }
 
 __device__ inline bool aborted(const Control* ctl) { return *reinterpret_cast<const volatile int*>(&ctl->abort_flag) != 0; }
@@ -109,7 +117,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
     uint8_t* const stages = smem;
     uint8_t* const qslots = smem + (size_t)nst * kStageBytes;
     TailSmem<kTailThreads>* const tsm =
-        reinterpret_cast<TailSmem<kTailThreads>*>(qslots + (size_t)nst * kQSlotBytes);
+        reinterpret_cast<TailSmem<kTailThreads>*>(qslots + (size_t)kQSlots * kQSlotBytes);
     Control* const ctl = reinterpret_cast<Control*>(reinterpret_cast<uint8_t*>(tsm) + ((sizeof(TailSmem<kTailThreads>) + 15) & ~size_t(15)));
 
     const LayerDev& L = p.L;
@@ -124,6 +132,10 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             ptx::mbar_init(ptx::smem_u32(&ctl->empty[s]), kConsumerWarps);
             ptx::mbar_init(ptx::smem_u32(&ctl->xfull[s]), kConsumerWarps);
         }
+        for (int s = 0; s < kQSlots; ++s) {
+            ptx::mbar_init(ptx::smem_u32(&ctl->qfull[s]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctl->qempty[s]), kConsumerWarps);
+        }
         ctl->abort_flag = 0;
         ctl->last_flag = 0;
         ctl->wait_ok = 1;
@@ -131,6 +143,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         ptx::fence_proxy_async();
     }
     __syncthreads();
+    if (tid == 0) { MKV_TR(0); MKV_TR_SET(6, 0); }
 
     if (warp == kConsumerWarps) {
         // ================================ producer =====================================
@@ -140,6 +153,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             uint32_t issued = 0;       // bit s: a copy into stage s may still be in flight
             uint32_t issued_par = 0;   // parity its full barrier completes with
             bool ok = true;
+            int qcount = 0;            // items that had at least one tile (and therefore a query slot)
             auto acquire = [&]() -> bool {
                 if (!wait_or_abort(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl)) {
                     if (!aborted(ctl)) note_timeout(p, ctl);
@@ -169,14 +183,27 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
                     const uint8_t* kb = (tr.seg == 0 ? L.Kp : L.Kd) + off;
                     const uint8_t* vb = (tr.seg == 0 ? L.Vp : L.Vd) + off;
                     const uint32_t bytes = (uint32_t)tr.cnt * kRowB;
-                    ptx::mbar_arrive_expect_tx(fb, 2u * bytes + (first ? (uint32_t)G * kRowB : 0u));
-                    ptx::bulk_g2s(dstK, kb, bytes, fb);
-                    ptx::bulk_g2s(dstK + kTileBytes, vb, bytes, fb);
                     if (first) {
+                        // the unit's G query rows, one padded row each, into the next query slot
+                        const int qi = qcount & 1;
+                        if (!wait_or_abort(ptx::smem_u32(&ctl->qempty[qi]), (uint32_t)(((qcount >> 1) & 1) ^ 1), ctl)) {
+                            if (!aborted(ctl)) note_timeout(p, ctl);
+                            ok = false;
+                            break;
+                        }
+                        const uint32_t qb = ptx::smem_u32(&ctl->qfull[qi]);
                         const uint8_t* qsrc = reinterpret_cast<const uint8_t*>(p.q) +
                                               ((size_t)b * p.q_heads + (size_t)g * G) * kRowB;
-                        ptx::bulk_g2s(ptx::smem_u32(qslots + (size_t)stage * kQSlotBytes), qsrc, (uint32_t)G * kRowB, fb);
+                        ptx::mbar_arrive_expect_tx(qb, (uint32_t)G * kRowB);
+                        for (int h = 0; h < G; ++h)
+                            ptx::bulk_g2s(ptx::smem_u32(qslots + (size_t)qi * kQSlotBytes + (size_t)h * kQRowB),
+                                          qsrc + (size_t)h * kRowB, kRowB, qb);
+                        ++qcount;
                     }
+                    ptx::mbar_arrive_expect_tx(fb, 2u * bytes);
+                    ptx::bulk_g2s(dstK, kb, bytes, fb);
+                    ptx::bulk_g2s(dstK + kTileBytes, vb, bytes, fb);
+                    if (qcount == 1 && first) MKV_TR(1);
                     issued |= 1u << stage;
                     issued_par = (issued_par & ~(1u << stage)) | (phase << stage);
                     first = 0;
@@ -209,15 +236,14 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         int xcount = 0;
         float oacc[8][4];              // O^T: [16-dim block][dim 0-7 | 8-15 x head pair]
         float m_run = kNegBig, l_run = 0.f;
-        uint32_t qa[8][2];
+        int qcount = 0;
+        const uint8_t* qs = qslots;    // this lane's place in the current query slot
         const int head = lane >> 2, tk0 = 2 * (lane & 3);
         const int mi = lane >> 3, rr = lane & 7;
         const int blk0 = warp * 16;
         float* lg = L.logit;           // this lane's head row of the unit's logit scratch
 #pragma unroll
         for (int j = 0; j < 8; ++j) { oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f; }
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) { qa[ks][0] = qa[ks][1] = 0u; }
 
         for (;;) {
             if (!wait_or_abort(ptx::smem_u32(&ctl->full[stage]), phase, ctl)) {
@@ -225,7 +251,8 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
                 break;
             }
             const StageMeta mt = ctl->meta[stage];
-            if (mt.kind == kEntryEnd) break;
+            if (warp == 0 && lane == 0 && xcount == 0 && mt.first) MKV_TR(2);
+            if (mt.kind == kEntryEnd) { if (warp == 0 && lane == 0) MKV_TR(3); break; }
             uint8_t* const sK = stages + (size_t)stage * kStageBytes;
             uint8_t* const sV = sK + kTileBytes;
             if (mt.first) {
@@ -237,14 +264,12 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
                     lg = L.logit + ((size_t)b * p.q_heads + (size_t)g * G + min(head, G - 1)) * p.lstride;
                 }
                 if (mt.kind == kEntryTile) {
-                    const uint8_t* qs = qslots + (size_t)stage * kQSlotBytes + (size_t)min(head, G - 1) * kRowB + tk0 * 2;
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t x0 = *reinterpret_cast<const uint32_t*>(qs + 32 * ks);
-                        const uint32_t x1 = *reinterpret_cast<const uint32_t*>(qs + 32 * ks + 16);
-                        qa[ks][0] = head < G ? x0 : 0u;
-                        qa[ks][1] = head < G ? x1 : 0u;
+                    const int qi = qcount & 1;
+                    if (!wait_or_abort(ptx::smem_u32(&ctl->qfull[qi]), (uint32_t)((qcount >> 1) & 1), ctl)) {
+                        if (lane == 0 && !aborted(ctl)) note_timeout(p, ctl);
+                        break;
                     }
+                    qs = qslots + (size_t)qi * kQSlotBytes + (size_t)head * kQRowB + tk0 * 2;
                 }
             }
             if (mt.kind == kEntryTile) {
@@ -269,8 +294,12 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
                     for (int ks = 0; ks < 8; ++ks) {
                         uint32_t b00, b01, b10, b11;
                         ptx::ldmatrix_x4(kbase + (uint32_t)(((2 * ks + (mi & 1)) ^ rr) << 4), b00, b01, b10, b11);
-                        ptx::mma_bf16(sacc[0], qa[ks][0], 0u, qa[ks][1], 0u, b00, b01);
-                        ptx::mma_bf16(sacc[1], qa[ks][0], 0u, qa[ks][1], 0u, b10, b11);
+                        // A fragment: this head's query elements (rows past G are zero)
+                        uint32_t qa0 = *reinterpret_cast<const uint32_t*>(qs + 32 * ks);
+                        uint32_t qa1 = *reinterpret_cast<const uint32_t*>(qs + 32 * ks + 16);
+                        if (head >= G) { qa0 = 0u; qa1 = 0u; }
+                        ptx::mma_bf16(sacc[0], qa0, 0u, qa1, 0u, b00, b01);
+                        ptx::mma_bf16(sacc[1], qa0, 0u, qa1, 0u, b10, b11);
                     }
                     // ---------------- online softmax in registers (fp32) -------------------------
                     float s[4] = {sacc[0][0], sacc[0][1], sacc[1][0], sacc[1][1]};
@@ -337,6 +366,10 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
                     oA[16 * j] = oacc[j][0]; oB[16 * j] = oacc[j][1];
                     oA[16 * j + 8] = oacc[j][2]; oB[16 * j + 8] = oacc[j][3];
                 }
+                if (!mt.first) {     // the item had tiles: its query slot is free again
+                    if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->qempty[qcount & 1]));
+                    ++qcount;
+                }
                 const int xs = xcount % nst;
                 if (warp == 0 && lane == 0) { ctl->xq[xs].stage = stage; ctl->xq[xs].unit = mt.unit; ctl->xq[xs].item = mt.item; }
                 ptx::fence_proxy_async();
@@ -390,11 +423,14 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             if ((tt & 31) == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->empty[ref.stage]));
             if (tt == 0) ctl->last_flag = (atomicAdd(&L.ticket[u], 1) == L.unit_nparts[u] - 1);
             bar_sync(1, kTailThreads);
+            if (tt == 0) MKV_TR(4);
             if (ctl->last_flag) {
+                if (tt == 0) MKV_TR_ADD(6, 1);
                 __threadfence();
                 unit_tail<__nv_bfloat16, kTailThreads, 1>(p, u, *tsm, tt);
             }
             bar_sync(1, kTailThreads);
+            if (tt == 0) MKV_TR(5);
         }
     }
 }
@@ -402,6 +438,12 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
 int g_stages = 3;
 
 }  // namespace
+
+#ifdef MKV_TRACE
+extern "C" __attribute__((visibility("default"))) int mkv_debug_trace(unsigned long long* host, int n) {
+    return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(unsigned long long) * n);
+}
+#endif
 
 bool mma_supported(int kv_dtype, int head_dim, int group) {
     return kv_dtype == 0 && head_dim == 128 && group >= 1 && group <= kMaxGroup;

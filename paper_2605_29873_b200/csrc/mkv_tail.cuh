@@ -93,6 +93,7 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid) {
             r.ps = *reinterpret_cast<const int4*>(pos + i0);
         }
     };
+    if (tid == 0) MKV_TR(8);
     Tok tk;
     if (dec) load_tok(4 * tid, tk);
     for (int e0 = 0; e0 < P * kMaxGroup; e0 += NT) {
@@ -113,7 +114,9 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid) {
             if (lane == 0) sm.snew[h] = a * p.scale_log2;
         }
     }
+    if (tid == 0) MKV_TR(9);
     bar_sync(BAR, NT);
+    if (tid == 0) MKV_TR(10);
 
     // ---- 1. combine -----------------------------------------------------------------------
     if (tid < G) {
@@ -152,6 +155,7 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid) {
             else reinterpret_cast<__nv_bfloat16*>(p.out)[obase + idx] = __float2bfloat16_rn(acc);
         }
     }
+    if (tid == 0) MKV_TR(11);
     if (!dec) {
         if (tid == 0) L.ticket[u] = 0;
         return;
@@ -209,6 +213,7 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid) {
             }
         }
     }
+    if (tid == 0) MKV_TR(12);
     if (tid == NT - 1) {                              // the fresh token sits (virtually) in slot n_old
         if (key_new < best_key) { best_key = key_new; best_slot = n_old; }
         if (L.abar) L.abar[(size_t)u * cap + n_old] = ab_new;
@@ -244,6 +249,7 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid) {
             L.ev_pos[(size_t)u * cap] = (int32_t)(unsigned)(kk & 0xffffffffu);
             L.ev_score[(size_t)u * cap] = __uint_as_float((unsigned)(kk >> 32));
         }
+        if (tid == 0) MKV_TR(13);
         // ---- 5a. the fresh row lands in the hole -----------------------------------------
         if (e != n_old) {
             if (warp == 0) store_row_swizzled(L.Kd, ubase, rowb, knew, e, lane);
