@@ -117,7 +117,7 @@ __device__ inline void bar_sync(int id, int nthreads) {
 // Optional per-CTA timestamps (diagnostic builds only: compile with -DMKV_TRACE).  Slot i of
 // CTA c is g_trace[c * 16 + i]; mkv_debug_trace() copies the array to the host.
 #ifdef MKV_TRACE
-extern __device__ unsigned long long g_trace[kMaxCtas * 16];
+static __device__ unsigned long long g_trace[kMaxCtas * 16];   // one copy per translation unit
 __device__ inline unsigned long long trace_now() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));

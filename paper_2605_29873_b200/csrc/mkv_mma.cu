@@ -39,9 +39,6 @@
 #include "mkv_tail.cuh"
 
 namespace mkv {
-#ifdef MKV_TRACE
-__device__ unsigned long long g_trace[kMaxCtas * 16];
-#endif
 namespace {
 
 constexpr int kRowB = 256;                                // 128 bf16
@@ -153,6 +150,9 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             uint32_t issued = 0;       // bit s: a copy into stage s may still be in flight
             uint32_t issued_par = 0;   // parity its full barrier completes with
             bool ok = true;
+            // K and V are read exactly once per step: let them leave L2 first, so that the
+            // step's scratch (logits, partials) and the scores stay resident for the tails
+            const unsigned long long stream_policy = ptx::l2_policy_evict_first();
             int qcount = 0;            // items that had at least one tile (and therefore a query slot)
             auto acquire = [&]() -> bool {
                 if (!wait_or_abort(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl)) {
@@ -201,8 +201,8 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
                         ++qcount;
                     }
                     ptx::mbar_arrive_expect_tx(fb, 2u * bytes);
-                    ptx::bulk_g2s(dstK, kb, bytes, fb);
-                    ptx::bulk_g2s(dstK + kTileBytes, vb, bytes, fb);
+                    ptx::bulk_g2s_hint(dstK, kb, bytes, fb, stream_policy);
+                    ptx::bulk_g2s_hint(dstK + kTileBytes, vb, bytes, fb, stream_policy);
                     if (qcount == 1 && first) MKV_TR(1);
                     issued |= 1u << stage;
                     issued_par = (issued_par & ~(1u << stage)) | (phase << stage);

@@ -240,6 +240,8 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid) {
             if (ok < best_key) { best_key = ok; best_slot = os; }
         }
         if (lane == 0) { sm.red_key[warp] = best_key; sm.red_slot[warp] = best_slot; }
+        if (tid == 0) MKV_TR(14);
+        if (tid == NT - 1) MKV_TR(15);
         bar_sync(BAR, NT);   // also orders every score write before the stores below
         unsigned long long kk = sm.red_key[0];
         int e = sm.red_slot[0];
