@@ -199,6 +199,12 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
                             ptx::bulk_g2s(ptx::smem_u32(qslots + (size_t)qi * kQSlotBytes + (size_t)h * kQRowB),
                                           qsrc + (size_t)h * kRowB, kRowB, qb);
                         ++qcount;
+                        if (dec) {   // the tail will want the fresh token's rows: bring them into L2 now
+                            const uint8_t* kn = reinterpret_cast<const uint8_t*>(p.k_new) + (size_t)u * kRowB;
+                            const uint8_t* vn = reinterpret_cast<const uint8_t*>(p.v_new) + (size_t)u * kRowB;
+                            ptx::prefetch_l2(kn); ptx::prefetch_l2(kn + 128);
+                            ptx::prefetch_l2(vn); ptx::prefetch_l2(vn + 128);
+                        }
                     }
                     ptx::mbar_arrive_expect_tx(fb, 2u * bytes);
                     ptx::bulk_g2s_hint(dstK, kb, bytes, fb, stream_policy);
@@ -427,7 +433,9 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             if (ctl->last_flag) {
                 if (tt == 0) MKV_TR_ADD(6, 1);
                 __threadfence();
-                unit_tail<__nv_bfloat16, kTailThreads, 1>(p, u, *tsm, tt);
+                const TailJob job = load_tail_job(L, u);
+                if (G <= 4) unit_tail<__nv_bfloat16, kTailThreads, 1, 4>(p, job, *tsm, tt);
+                else unit_tail<__nv_bfloat16, kTailThreads, 1, 8>(p, job, *tsm, tt);
             }
             bar_sync(1, kTailThreads);
             if (tt == 0) MKV_TR(5);

@@ -156,7 +156,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
         __syncthreads();
         if (s_last) {
             __threadfence();
-            unit_tail<T, kSimtThreads, 1>(p, u, tsm, tid);
+            unit_tail<T, kSimtThreads, 1, (G <= 4 ? 4 : 8)>(p, load_tail_job(L, u), tsm, tid);
         }
         __syncthreads();
     }

@@ -59,43 +59,121 @@ __device__ inline void store_row_swizzled(uint8_t* pool, size_t unit_base, int r
     for (int c = lane; c < chunks; c += 32) d[c ^ (dst & 7)] = __ldg(&s[c]);
 }
 
-template <typename T, int NT, int BAR>
-__device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid) {
+// N consecutive elements of type T as floats, fetched with one vector load.
+template <typename T, int N>
+__device__ inline void load_elems(const T* ptr, float (&f)[N]) {
+    static_assert(N == 2 || N == 4, "two or four elements");
+    if constexpr (sizeof(T) * N == 16) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(ptr));
+        const T* e = reinterpret_cast<const T*>(&v);
+#pragma unroll
+        for (int i = 0; i < N; ++i) f[i] = to_f32(e[i]);
+    } else if constexpr (sizeof(T) * N == 8) {
+        const uint2 v = __ldg(reinterpret_cast<const uint2*>(ptr));
+        const T* e = reinterpret_cast<const T*>(&v);
+#pragma unroll
+        for (int i = 0; i < N; ++i) f[i] = to_f32(e[i]);
+    } else {
+        const uint32_t v = __ldg(reinterpret_cast<const uint32_t*>(ptr));
+        const T* e = reinterpret_cast<const T*>(&v);
+#pragma unroll
+        for (int i = 0; i < N; ++i) f[i] = to_f32(e[i]);
+    }
+}
+
+// What a tail needs to know about its unit.  Whoever takes the last ticket loads it (the
+// loads overlap that thread's other work) and hands it over.
+struct TailJob { int u, P, part0, n_dec, t; };
+
+__device__ inline TailJob load_tail_job(const LayerDev& L, int u) {
+    TailJob j;
+    j.u = u; j.P = L.unit_nparts[u]; j.part0 = L.unit_part0[u]; j.n_dec = L.n_dec[u]; j.t = L.unit_step[u];
+    return j;
+}
+
+__device__ inline void store_out4(const Params& p, size_t idx, float4 v) {
+    if (p.out_f32) {
+        *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + idx) = v;
+    } else {
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+        uint2 pk;
+        pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+        pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + idx) = pk;
+    }
+}
+
+// GB: compile-time bound of the group size G (4 or 8); it sizes the register staging.
+template <typename T, int NT, int BAR, int GB>
+__device__ void unit_tail(const Params& p, const TailJob& job, TailSmem<NT>& sm, int tid) {
     const LayerDev& L = p.L;
+    const int u = job.u;
     const int G = p.group, D = p.head_dim, cap = p.cap, ls = p.lstride;
     const int rowb = D * (int)sizeof(T);
     const int b = u / p.kv_heads, g = u - b * p.kv_heads;
-    const int P = L.unit_nparts[u], part0 = L.unit_part0[u];
+    const int P = job.P, part0 = job.part0;
     const bool dec = (p.mode == kModeDecode);
-    const int n_old = min(L.n_dec[u], dec ? cap - 1 : cap);
+    const int n_old = min(job.n_dec, dec ? cap - 1 : cap);
     const int n = dec ? n_old + 1 : n_old;
-    const int t = L.unit_step[u];     // read before the first barrier: thread 0 advances it below
+    const int t = job.t;
     const int lane = tid & 31, warp = tid >> 5;
     constexpr int NW = NT / 32;
+    constexpr int TW = GB <= 4 ? 4 : 2;                 // tokens per thread and pass (one 16- or 8-byte vector)
+    constexpr int TV = 1;                               // token vectors per thread loaded up front
+    constexpr int PB = GB <= 4 ? 2 : 1;                 // partials staged in registers up front
+    constexpr int LB = 4;                               // partials fetched per trip after those
+    constexpr int OCB = (GB * 32 + NT - 1) / NT;        // float4 output elements per thread (bound)
     const T* qrow = reinterpret_cast<const T*>(p.q) + ((size_t)b * p.q_heads + (size_t)g * G) * D;
     const T* knew = reinterpret_cast<const T*>(p.k_new) + (size_t)u * D;
     const T* vnew = reinterpret_cast<const T*>(p.v_new) + (size_t)u * D;
     float* score = L.score + (size_t)u * ls;
     int32_t* pos = L.pos + (size_t)u * ls;
     const float* lg = L.logit + ((size_t)b * p.q_heads + (size_t)g * G) * ls;
+    const float* po_base = L.part_o + (size_t)part0 * G * D;
+    const size_t pstride = (size_t)G * D;
+    const int ne = G * D / 4;                           // float4 elements of one partial / of `out`
+    if (tid == 0) MKV_TR(8);
 
-    // Everything below is latency: a handful of dependent trips to L2.  So every load that
-    // does not need the softmax statistics is issued first, in one batch: the partials'
-    // (m, l), the fresh token's dot products, and this thread's first four tokens' logits,
-    // scores and position ids (as 16-byte vectors).
-    struct Tok { float4 lgv[kMaxGroup]; float4 sc; int4 ps; };
+    // Everything below is latency: a few dependent trips to L2.  So every load that does
+    // not need the softmax statistics is issued first, in one batch: this thread's tokens'
+    // logits, scores and position ids (one vector each), its share of the first partials'
+    // O, the fresh token's value and dot products, and the partials' (m, l).
+    struct Tok { float lgv[GB][TW]; float sc[TW]; int ps[TW]; };
+    auto load_vec = [&](const float* src, float (&dst)[TW]) {
+        if constexpr (TW == 4) {
+            const float4 v = __ldcg(reinterpret_cast<const float4*>(src));
+            dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+        } else {
+            const float2 v = __ldcg(reinterpret_cast<const float2*>(src));
+            dst[0] = v.x; dst[1] = v.y;
+        }
+    };
     auto load_tok = [&](int i0, Tok& r) {
         if (i0 < n_old) {
 #pragma unroll
-            for (int h = 0; h < kMaxGroup; ++h)
-                if (h < G) r.lgv[h] = __ldcg(reinterpret_cast<const float4*>(lg + (size_t)h * ls + i0));
-            r.sc = *reinterpret_cast<const float4*>(score + i0);
-            r.ps = *reinterpret_cast<const int4*>(pos + i0);
+            for (int h = 0; h < GB; ++h)
+                if (h < G) load_vec(lg + (size_t)h * ls + i0, r.lgv[h]);
+            load_vec(score + i0, r.sc);
+            float pf[TW];
+            load_vec(reinterpret_cast<const float*>(pos + i0), pf);
+#pragma unroll
+            for (int j = 0; j < TW; ++j) r.ps[j] = __float_as_int(pf[j]);
         }
     };
-    if (tid == 0) MKV_TR(8);
-    Tok tk;
-    if (dec) load_tok(4 * tid, tk);
+    Tok tk[TV];
+    if (dec) {
+#pragma unroll
+        for (int v = 0; v < TV; ++v) load_tok(TW * (tid + v * NT), tk[v]);
+    }
+    float4 po[PB][OCB];
+#pragma unroll
+    for (int q = 0; q < PB; ++q)
+#pragma unroll
+        for (int c = 0; c < OCB; ++c) {
+            const int e = tid + c * NT;
+            po[q][c] = (q < P && e < ne) ? __ldcg(reinterpret_cast<const float4*>(po_base + (size_t)q * pstride) + e)
+                                          : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
     for (int e0 = 0; e0 < P * kMaxGroup; e0 += NT) {
         const int e = e0 + tid, q = e / kMaxGroup, h = e - q * kMaxGroup;
         if (q < P && h < G) {
@@ -104,11 +182,27 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid) {
             sm.pl[q][h] = ml.y;
         }
     }
-    // ---- 0. logit of the fresh token ------------------------------------------------------
+    // ---- 0. the fresh token: its value row and its logit (lane l holds D/32 consecutive elements)
+    float vn[OCB][4];
     if (dec) {
+#pragma unroll
+        for (int c = 0; c < OCB; ++c) {
+            const int e = tid + c * NT;
+            if (e < ne) load_elems<T, 4>(vnew + (4 * e) % D, vn[c]);
+        }
         for (int h = warp; h < G; h += NW) {
             float a = 0.f;
-            for (int e = lane; e < D; e += 32) a = fmaf(to_f32(qrow[(size_t)h * D + e]), to_f32(knew[e]), a);
+            if (D == 128) {
+                float qv[4], kv[4];
+                load_elems<T, 4>(qrow + (size_t)h * D + 4 * lane, qv);
+                load_elems<T, 4>(knew + 4 * lane, kv);
+                a = fmaf(qv[0], kv[0], fmaf(qv[1], kv[1], fmaf(qv[2], kv[2], qv[3] * kv[3])));
+            } else {
+                float qv[2], kv[2];
+                load_elems<T, 2>(qrow + (size_t)h * D + 2 * lane, qv);
+                load_elems<T, 2>(knew + 2 * lane, kv);
+                a = fmaf(qv[0], kv[0], qv[1] * kv[1]);
+            }
 #pragma unroll
             for (int off = 16; off; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
             if (lane == 0) sm.snew[h] = a * p.scale_log2;
@@ -135,31 +229,60 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid) {
         sm.invL[tid] = Lsum > 0.f ? 1.0f / Lsum : 0.f;
     }
     bar_sync(BAR, NT);
-    {
-        const size_t obase = ((size_t)b * p.q_heads + (size_t)g * G) * D;
-        const float* po = L.part_o + (size_t)part0 * G * D;
-        const size_t pstride = (size_t)G * D;
-        for (int idx = tid; idx < G * D; idx += NT) {
-            const int h = idx / D;
-            float acc = dec ? to_f32(vnew[idx - h * D]) * sm.wnew[h] : 0.f;
-            int q = 0;
-            for (; q + 4 <= P; q += 4) {
-                const float v0 = __ldcg(po + (size_t)q * pstride + idx), v1 = __ldcg(po + (size_t)(q + 1) * pstride + idx);
-                const float v2 = __ldcg(po + (size_t)(q + 2) * pstride + idx), v3 = __ldcg(po + (size_t)(q + 3) * pstride + idx);
-                acc = fmaf(v0, sm.w[q][h], acc); acc = fmaf(v1, sm.w[q + 1][h], acc);
-                acc = fmaf(v2, sm.w[q + 2][h], acc); acc = fmaf(v3, sm.w[q + 3][h], acc);
-            }
-            for (; q < P; ++q) acc = fmaf(__ldcg(po + (size_t)q * pstride + idx), sm.w[q][h], acc);
-            acc *= sm.invL[h];
-            if (p.out_f32) reinterpret_cast<float*>(p.out)[obase + idx] = acc;
-            else reinterpret_cast<__nv_bfloat16*>(p.out)[obase + idx] = __float2bfloat16_rn(acc);
+    // out, part 1: the fresh token and the partials staged in registers
+    const size_t obase = ((size_t)b * p.q_heads + (size_t)g * G) * D;
+    float4 oacc[OCB];
+#pragma unroll
+    for (int c = 0; c < OCB; ++c) {
+        const int e = tid + c * NT;
+        const int h = min((4 * e) / D, G - 1);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (dec) {
+            const float wn = sm.wnew[h];
+            acc = make_float4(vn[c][0] * wn, vn[c][1] * wn, vn[c][2] * wn, vn[c][3] * wn);
         }
+#pragma unroll
+        for (int q = 0; q < PB; ++q) {
+            if (q < P) {
+                const float w = sm.w[q][h];
+                acc.x = fmaf(po[q][c].x, w, acc.x); acc.y = fmaf(po[q][c].y, w, acc.y);
+                acc.z = fmaf(po[q][c].z, w, acc.z); acc.w = fmaf(po[q][c].w, w, acc.w);
+            }
+        }
+        oacc[c] = acc;
     }
-    if (tid == 0) MKV_TR(11);
+    // out, part 2: the remaining partials, several per trip, then the store
+    auto finish_out = [&]() {
+#pragma unroll
+        for (int c = 0; c < OCB; ++c) {
+            const int e = tid + c * NT;
+            if (e >= ne) continue;
+            const int h = (4 * e) / D;
+            float4 acc = oacc[c];
+            for (int q0 = PB; q0 < P; q0 += LB) {
+                float4 v[LB];
+#pragma unroll
+                for (int j = 0; j < LB; ++j)
+                    v[j] = (q0 + j < P) ? __ldcg(reinterpret_cast<const float4*>(po_base + (size_t)(q0 + j) * pstride) + e)
+                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int j = 0; j < LB; ++j) {
+                    const float w = (q0 + j < P) ? sm.w[q0 + j][h] : 0.f;
+                    acc.x = fmaf(v[j].x, w, acc.x); acc.y = fmaf(v[j].y, w, acc.y);
+                    acc.z = fmaf(v[j].z, w, acc.z); acc.w = fmaf(v[j].w, w, acc.w);
+                }
+            }
+            const float il = sm.invL[h];
+            store_out4(p, obase + 4 * (size_t)e, make_float4(acc.x * il, acc.y * il, acc.z * il, acc.w * il));
+        }
+    };
     if (!dec) {
+        finish_out();
+        if (tid == 0) MKV_TR(11);
         if (tid == 0) L.ticket[u] = 0;
         return;
     }
+    if (tid == 0) MKV_TR(11);
 
     // ---- 2./3. probabilities, head mean, momentum update ---------------------------------
     const int k = max(0, n - p.budget);
@@ -171,48 +294,52 @@ __device__ void unit_tail(const Params& p, int u, TailSmem<NT>& sm, int tid) {
     const unsigned long long key_new = ((unsigned long long)__float_as_uint(ab_new) << 32) | (unsigned)t;
     unsigned long long best_key = ~0ull;
     int best_slot = -1;
-    float Mh[kMaxGroup], iLh[kMaxGroup];
+    auto process_tok = [&](int i0, const Tok& r) {
+        if (i0 >= n_old) return;
+        float ab[TW], nw[TW];
 #pragma unroll
-    for (int h = 0; h < kMaxGroup; ++h) { Mh[h] = h < G ? sm.M[h] : 0.f; iLh[h] = h < G ? sm.invL[h] : 0.f; }
-    for (int base = 0; base < n_old; base += 4 * NT) {
-        const int i0 = base + 4 * tid;
-        if (base > 0) load_tok(i0, tk);
-        if (i0 < n_old) {
-            float ab[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int j = 0; j < TW; ++j) ab[j] = 0.f;
 #pragma unroll
-            for (int h = 0; h < kMaxGroup; ++h) {
-                if (h < G) {
-                    ab[0] = fmaf(fast_exp2(tk.lgv[h].x - Mh[h]), iLh[h], ab[0]);
-                    ab[1] = fmaf(fast_exp2(tk.lgv[h].y - Mh[h]), iLh[h], ab[1]);
-                    ab[2] = fmaf(fast_exp2(tk.lgv[h].z - Mh[h]), iLh[h], ab[2]);
-                    ab[3] = fmaf(fast_exp2(tk.lgv[h].w - Mh[h]), iLh[h], ab[3]);
-                }
-            }
-            const float old[4] = {tk.sc.x, tk.sc.y, tk.sc.z, tk.sc.w};
-            const int ps[4] = {tk.ps.x, tk.ps.y, tk.ps.z, tk.ps.w};
-            float nw[4];
+        for (int h = 0; h < GB; ++h) {
+            if (h < G) {
+                const float Mh = sm.M[h], iLh = sm.invL[h];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                ab[j] *= inv_g;
-                nw[j] = fmaf(p.beta, old[j], ab[j]);
-            }
-            if (i0 + 4 <= n_old) {
-                *reinterpret_cast<float4*>(score + i0) = make_float4(nw[0], nw[1], nw[2], nw[3]);
-            } else {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) if (i0 + j < n_old) score[i0 + j] = nw[j];
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if (i0 + j < n_old) {
-                    if (L.abar) L.abar[(size_t)u * cap + i0 + j] = ab[j];
-                    const unsigned long long key = ((unsigned long long)__float_as_uint(nw[j]) << 32) | (unsigned)ps[j];
-                    if (k > 1) keys[i0 + j] = key;
-                    if (key < best_key) { best_key = key; best_slot = i0 + j; }
-                }
+                for (int j = 0; j < TW; ++j) ab[j] = fmaf(fast_exp2(r.lgv[h][j] - Mh), iLh, ab[j]);
             }
         }
+#pragma unroll
+        for (int j = 0; j < TW; ++j) {
+            ab[j] *= inv_g;
+            nw[j] = fmaf(p.beta, r.sc[j], ab[j]);
+        }
+        if (i0 + TW <= n_old) {
+            if constexpr (TW == 4) *reinterpret_cast<float4*>(score + i0) = make_float4(nw[0], nw[1], nw[2], nw[3]);
+            else *reinterpret_cast<float2*>(score + i0) = make_float2(nw[0], nw[1]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < TW; ++j) if (i0 + j < n_old) score[i0 + j] = nw[j];
+        }
+#pragma unroll
+        for (int j = 0; j < TW; ++j) {
+            if (i0 + j < n_old) {
+                if (L.abar) L.abar[(size_t)u * cap + i0 + j] = ab[j];
+                const unsigned long long key = ((unsigned long long)__float_as_uint(nw[j]) << 32) | (unsigned)r.ps[j];
+                if (k > 1) keys[i0 + j] = key;
+                if (key < best_key) { best_key = key; best_slot = i0 + j; }
+            }
+        }
+    };
+#pragma unroll
+    for (int v = 0; v < TV; ++v) process_tok(TW * (tid + v * NT), tk[v]);
+    // further passes; the rest of `out` travels with the first of them (one trip, not two)
+    bool out_done = false;
+    for (int base = TV * TW * NT; base < n_old; base += TW * NT) {
+        const int i0 = base + TW * tid;
+        load_tok(i0, tk[0]);
+        if (!out_done) { finish_out(); out_done = true; }
+        process_tok(i0, tk[0]);
     }
+    if (!out_done) finish_out();
     if (tid == 0) MKV_TR(12);
     if (tid == NT - 1) {                              // the fresh token sits (virtually) in slot n_old
         if (key_new < best_key) { best_key = key_new; best_slot = n_old; }
