@@ -124,6 +124,8 @@ struct mkv_ctx {
     int n_ctas_max; // persistent grid upper bound (SM count x resident CTAs per SM)
     bool use_mma;
     std::vector<char> prefilled;
+    std::vector<char> stepped;   // a step has run on the layer since its prefill
+    bool pdl;
     std::vector<int> n_items;
     std::vector<int> n_ctas;
     std::vector<std::vector<int32_t>> lens;   // per layer, per sequence
@@ -180,10 +182,14 @@ Params make_params(const mkv_ctx* c, int layer, const void* q, const void* k_new
     return p;
 }
 
-mkv_status launch_step(mkv_ctx* c, const Params& p, cudaStream_t st) {
-    cudaError_t e = c->use_mma ? launch_mma(p, st) : launch_simt(p, c->kv_dtype, st);
+mkv_status launch_step(mkv_ctx* c, int layer, const Params& p, cudaStream_t st) {
+    // The first step after a prefill must see the prefill's copies complete before it reads
+    // the pool; later steps may overlap their start with the previous kernel's end.
+    const bool overlap = c->pdl && c->stepped[layer];
+    cudaError_t e = c->use_mma ? launch_mma(p, st, overlap) : launch_simt(p, c->kv_dtype, st);
     if (e != cudaSuccess) return MKV_ERR_CUDA;
     c->launches += 1;
+    c->stepped[layer] = 1;
     return MKV_OK;
 }
 
@@ -263,6 +269,9 @@ mkv_status mkv_create(int layers, int q_heads, int kv_heads, int head_dim, int b
     if (const char* e = std::getenv("MKV_CTAS_PER_SM")) per_sm = std::max(1, std::min(16, std::atoi(e)));
     c->n_ctas_max = std::min(kMaxCtas, prop.multiProcessorCount * per_sm);
     c->prefilled.assign(layers, 0);
+    c->stepped.assign(layers, 0);
+    c->pdl = true;
+    if (const char* e = std::getenv("MKV_NO_OVERLAP")) c->pdl = std::atoi(e) == 0;
     c->n_items.assign(layers, 0);
     c->n_ctas.assign(layers, 0);
     c->lens.assign(layers, std::vector<int32_t>(batch, 0));
@@ -364,6 +373,7 @@ mkv_status mkv_prefill(mkv_ctx* c, int layer, const void* K, const void* V, cons
         c->launches += 1;
     }
     c->prefilled[layer] = 1;
+    c->stepped[layer] = 0;
     return MKV_OK;
 }
 
@@ -375,7 +385,7 @@ mkv_status mkv_decode_step(mkv_ctx* c, int layer, const void* q, const void* k_n
     DeviceGuard guard(c->device);
     if (!guard.ok) return MKV_ERR_CUDA;
     const Params p = make_params(c, layer, q, k_new, v_new, out, kModeDecode);
-    return launch_step(c, p, (cudaStream_t)stream);
+    return launch_step(c, layer, p, (cudaStream_t)stream);
 }
 
 mkv_status mkv_decode_step_host(mkv_ctx* c, int layer, const void* qh, const void* kh, const void* vh, void* outh,
@@ -393,7 +403,7 @@ mkv_status mkv_decode_step_host(mkv_ctx* c, int layer, const void* qh, const voi
     if (cudaMemcpyAsync(dk, kh, nk * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return MKV_ERR_CUDA;
     if (cudaMemcpyAsync(dv, vh, nk * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return MKV_ERR_CUDA;
     const Params p = make_params(c, layer, dq, dk, dv, dout, kModeDecode);
-    const mkv_status s = launch_step(c, p, st);
+    const mkv_status s = launch_step(c, layer, p, st);
     if (s != MKV_OK) return s;
     if (cudaMemcpyAsync(outh, dout, nq * os, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MKV_ERR_CUDA;
     return MKV_OK;
@@ -406,7 +416,7 @@ mkv_status mkv_attend_only(mkv_ctx* c, int layer, const void* q, void* out, void
     DeviceGuard guard(c->device);
     if (!guard.ok) return MKV_ERR_CUDA;
     const Params p = make_params(c, layer, q, nullptr, nullptr, out, kModeAttendOnly);
-    return launch_step(c, p, (cudaStream_t)stream);
+    return launch_step(c, layer, p, (cudaStream_t)stream);
 }
 
 mkv_status mkv_set_budget(mkv_ctx* c, int budget) {

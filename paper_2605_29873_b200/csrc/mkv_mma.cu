@@ -141,6 +141,8 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
     }
     __syncthreads();
     if (tid == 0) { MKV_TR(0); MKV_TR_SET(6, 0); }
+    // The next kernel of the stream may start as soon as SMs free up; it does its own waiting.
+    ptx::griddep_launch_dependents();
 
     if (warp == kConsumerWarps) {
         // ================================ producer =====================================
@@ -163,57 +165,78 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
                 return true;
             };
             auto advance = [&]() { if (++stage == nst) { stage = 0; phase ^= 1u; } };
+            auto issue_tile = [&](int u, int it, const TileRef& tr, int first) -> bool {
+                if (!acquire()) return false;
+                StageMeta& mt = ctl->meta[stage];
+                mt.kind = kEntryTile; mt.unit = u; mt.item = it; mt.seg = tr.seg; mt.row = tr.row;
+                mt.cnt = tr.cnt; mt.first = first;
+                const uint32_t fb = ptx::smem_u32(&ctl->full[stage]);
+                const uint32_t dstK = ptx::smem_u32(stages + (size_t)stage * kStageBytes);
+                const size_t off = ((size_t)u * (tr.seg == 0 ? p.max_prefill : p.cap) + tr.row) * kRowB;
+                const uint8_t* kb = (tr.seg == 0 ? L.Kp : L.Kd) + off;
+                const uint8_t* vb = (tr.seg == 0 ? L.Vp : L.Vd) + off;
+                const uint32_t bytes = (uint32_t)tr.cnt * kRowB;
+                ptx::mbar_arrive_expect_tx(fb, 2u * bytes);
+                ptx::bulk_g2s_hint(dstK, kb, bytes, fb, stream_policy);
+                ptx::bulk_g2s_hint(dstK + kTileBytes, vb, bytes, fb, stream_policy);
+                issued |= 1u << stage;
+                issued_par = (issued_par & ~(1u << stage)) | (phase << stage);
+                advance();
+                return true;
+            };
+            // the unit's G query rows, one padded row each, into the next query slot
+            auto issue_query = [&](int u) -> bool {
+                const int b = u / p.kv_heads, g = u - b * p.kv_heads;
+                const int qi = qcount & 1;
+                if (!wait_or_abort(ptx::smem_u32(&ctl->qempty[qi]), (uint32_t)(((qcount >> 1) & 1) ^ 1), ctl)) {
+                    if (!aborted(ctl)) note_timeout(p, ctl);
+                    return false;
+                }
+                const uint32_t qb = ptx::smem_u32(&ctl->qfull[qi]);
+                const uint8_t* qsrc = reinterpret_cast<const uint8_t*>(p.q) + ((size_t)b * p.q_heads + (size_t)g * G) * kRowB;
+                ptx::mbar_arrive_expect_tx(qb, (uint32_t)G * kRowB);
+                for (int h = 0; h < G; ++h)
+                    ptx::bulk_g2s(ptx::smem_u32(qslots + (size_t)qi * kQSlotBytes + (size_t)h * kQRowB),
+                                  qsrc + (size_t)h * kRowB, kRowB, qb);
+                ++qcount;
+                if (dec) {   // the tail will want the fresh token's rows: bring them into L2 now
+                    const uint8_t* kn = reinterpret_cast<const uint8_t*>(p.k_new) + (size_t)u * kRowB;
+                    const uint8_t* vn = reinterpret_cast<const uint8_t*>(p.v_new) + (size_t)u * kRowB;
+                    ptx::prefetch_l2(kn); ptx::prefetch_l2(kn + 128);
+                    ptx::prefetch_l2(vn); ptx::prefetch_l2(vn + 128);
+                }
+                return true;
+            };
+            // Before the dependency wait: only data no earlier kernel of the stream writes may be
+            // touched -- the work list and the frozen prefill pool.  So the first item's leading
+            // prefill tiles are already in flight while the previous step finishes its tails.
+            int pre = 0;
+            if (item_begin < item_end) {
+                const int4 v = __ldg(reinterpret_cast<const int4*>(&L.items[item_begin]));
+                const int lp = L.unit_lp[v.x];
+                const int tp = (lp + kTileRows - 1) / kTileRows;
+                const int t_end = min(v.y + v.z, tp);
+                for (int t = v.y; t < t_end && pre < nst && ok; ++t) {
+                    const TileRef tr = tile_ref(t, lp, 0);
+                    ok = issue_tile(v.x, item_begin, tr, pre == 0);
+                    if (ok) { if (pre == 0) MKV_TR(1); ++pre; }
+                }
+            }
+            ptx::griddep_wait();
             for (int it = item_begin; it < item_end && ok; ++it) {
                 const int4 v = __ldg(reinterpret_cast<const int4*>(&L.items[it]));
                 const int u = v.x, tile0 = v.y, ntiles = v.z;
                 const int lp = L.unit_lp[u];
                 const int n_old = min(L.n_dec[u], p.cap - (dec ? 1 : 0));
-                const int b = u / p.kv_heads, g = u - b * p.kv_heads;
-                int first = 1;
-                for (int t = tile0; t < tile0 + ntiles; ++t) {
+                int first = 1, t = tile0;
+                if (it == item_begin && pre > 0) { first = 0; t = tile0 + pre; }   // issued before the wait
+                // a non-empty first tile means the item has rows (empty decode tiles only trail)
+                if (tile_ref(tile0, lp, n_old).cnt > 0 && !(ok = issue_query(u))) break;
+                for (; t < tile0 + ntiles; ++t) {
                     const TileRef tr = tile_ref(t, lp, n_old);
                     if (tr.cnt == 0) continue;
-                    if (!(ok = acquire())) break;
-                    StageMeta& mt = ctl->meta[stage];
-                    mt.kind = kEntryTile; mt.unit = u; mt.item = it; mt.seg = tr.seg; mt.row = tr.row;
-                    mt.cnt = tr.cnt; mt.first = first;
-                    const uint32_t fb = ptx::smem_u32(&ctl->full[stage]);
-                    const uint32_t dstK = ptx::smem_u32(stages + (size_t)stage * kStageBytes);
-                    const size_t off = ((size_t)u * (tr.seg == 0 ? p.max_prefill : p.cap) + tr.row) * kRowB;
-                    const uint8_t* kb = (tr.seg == 0 ? L.Kp : L.Kd) + off;
-                    const uint8_t* vb = (tr.seg == 0 ? L.Vp : L.Vd) + off;
-                    const uint32_t bytes = (uint32_t)tr.cnt * kRowB;
-                    if (first) {
-                        // the unit's G query rows, one padded row each, into the next query slot
-                        const int qi = qcount & 1;
-                        if (!wait_or_abort(ptx::smem_u32(&ctl->qempty[qi]), (uint32_t)(((qcount >> 1) & 1) ^ 1), ctl)) {
-                            if (!aborted(ctl)) note_timeout(p, ctl);
-                            ok = false;
-                            break;
-                        }
-                        const uint32_t qb = ptx::smem_u32(&ctl->qfull[qi]);
-                        const uint8_t* qsrc = reinterpret_cast<const uint8_t*>(p.q) +
-                                              ((size_t)b * p.q_heads + (size_t)g * G) * kRowB;
-                        ptx::mbar_arrive_expect_tx(qb, (uint32_t)G * kRowB);
-                        for (int h = 0; h < G; ++h)
-                            ptx::bulk_g2s(ptx::smem_u32(qslots + (size_t)qi * kQSlotBytes + (size_t)h * kQRowB),
-                                          qsrc + (size_t)h * kRowB, kRowB, qb);
-                        ++qcount;
-                        if (dec) {   // the tail will want the fresh token's rows: bring them into L2 now
-                            const uint8_t* kn = reinterpret_cast<const uint8_t*>(p.k_new) + (size_t)u * kRowB;
-                            const uint8_t* vn = reinterpret_cast<const uint8_t*>(p.v_new) + (size_t)u * kRowB;
-                            ptx::prefetch_l2(kn); ptx::prefetch_l2(kn + 128);
-                            ptx::prefetch_l2(vn); ptx::prefetch_l2(vn + 128);
-                        }
-                    }
-                    ptx::mbar_arrive_expect_tx(fb, 2u * bytes);
-                    ptx::bulk_g2s_hint(dstK, kb, bytes, fb, stream_policy);
-                    ptx::bulk_g2s_hint(dstK + kTileBytes, vb, bytes, fb, stream_policy);
-                    if (qcount == 1 && first) MKV_TR(1);
-                    issued |= 1u << stage;
-                    issued_par = (issued_par & ~(1u << stage)) | (phase << stage);
+                    if (!(ok = issue_tile(u, it, tr, first))) break;
                     first = 0;
-                    advance();
                 }
                 if (!ok) break;
                 // the item's exchange entry: the consumers hand their state to the tail warps
@@ -237,6 +260,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         __syncwarp();
     } else if (warp < kConsumerWarps) {
         // ================================ consumers ====================================
+        ptx::griddep_wait();
         int stage = 0;
         uint32_t phase = 0;
         int xcount = 0;
@@ -387,6 +411,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         }
     } else {
         // ================================ tail warps ===================================
+        ptx::griddep_wait();
         const int tt = tid - kTailTid0;
         const int n_mine = item_end - item_begin;
         for (int x = 0; x < n_mine; ++x) {
@@ -462,10 +487,22 @@ cudaError_t mma_configure() {
     return cudaFuncSetAttribute(mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(g_stages));
 }
 
-cudaError_t launch_mma(const Params& p, cudaStream_t st) {
+// overlap: launch with programmatic stream serialization, i.e. this kernel's CTAs may start
+// while the previous kernel of the stream is still finishing; the kernel itself waits
+// (griddepcontrol.wait) before it touches anything an earlier kernel may write.
+cudaError_t launch_mma(const Params& p, cudaStream_t st, bool overlap) {
     if (p.L.n_ctas <= 0) return cudaSuccess;
-    mma_kernel<<<p.L.n_ctas, kThreads, smem_bytes(g_stages), st>>>(p, g_stages);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.L.n_ctas);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem_bytes(g_stages);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, mma_kernel, p, g_stages);
 }
 
 }  // namespace mkv

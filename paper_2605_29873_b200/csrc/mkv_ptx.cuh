@@ -77,6 +77,11 @@ __device__ inline unsigned long long l2_policy_evict_last() {
     return pol;
 }
 
+// Programmatic dependent launch: let the next kernel of the stream start early / wait until
+// every earlier kernel of the stream has completed and its writes are visible.
+__device__ inline void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ inline void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ inline void prefetch_l2(const void* p) {
     asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
 }
