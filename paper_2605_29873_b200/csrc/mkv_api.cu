@@ -1,5 +1,5 @@
-// C ABI of the Moment-KV decode library: argument checks, workspace carving, the static
-// work list, launches.  All device work is in the kernels; nothing here computes any
+// C ABI of the Moment-KV decode library: argument checks, workspace carving, the CTAs'
+// start table, launches.  All device work is in the kernels; nothing here computes any
 // step of the method on the host.
 #include <algorithm>
 #include <cmath>
@@ -22,13 +22,18 @@ inline int round4(int a) { return (a + 3) / 4 * 4; }
 inline int elem_size(int dt) { return dt == MKV_BF16 ? 2 : 4; }
 
 struct LayerOff {
-    size_t Kp, Vp, Kd, Vd, score, pos, n_dec, logit, abar, n_prev, ev_k, ev_pos, ev_score, items, cta_item0,
-        unit_lp, unit_part0, unit_nparts, part_o, part_ml, ticket, unit_step, keys, list_a, list_b, end;
+    size_t Kp, Vp, Kd, Vd, score, pos, n_dec, abar, n_prev, ev_k, ev_pos, ev_score, cta_unit0, cta_head0,
+        cta_headn, unit_lp, unit_next0, next, done, nslots, unit_step, end;
 };
+// Scratch that lives for one step only, shared by all layers of the context (calls on a
+// context are ordered on one stream, and a step touches it only after every earlier kernel
+// of the stream has completed).
+struct ScratchOff { size_t logit, part_o, part_ml, keys, list_a, list_b, end; };
 struct Layout {
-    int units, cap, rowb, max_items, lstride;
-    size_t status, stage_q, stage_k, stage_v, stage_out, layer0, layer_bytes, total;
-    LayerOff lo;  // offsets relative to the layer base
+    int units, cap, rowb, lstride;
+    size_t status, stage_q, stage_k, stage_v, stage_out, scratch0, scratch_bytes, layer0, layer_bytes, total;
+    ScratchOff so;  // offsets relative to the scratch base
+    LayerOff lo;    // offsets relative to the layer base
 };
 
 bool make_layout(int layers, int batch, int q_heads, int kv_heads, int head_dim, int budget, int max_prefill,
@@ -38,15 +43,13 @@ bool make_layout(int layers, int batch, int q_heads, int kv_heads, int head_dim,
     if (head_dim != 64 && head_dim != 128) return false;
     if (kv_dtype != MKV_BF16 && kv_dtype != MKV_F32) return false;
     const int G = q_heads / kv_heads;
-    if (G > kMaxGroup) return false;
+    if (G > 16) return false;
     if ((long long)budget + 1 > (1 << 24) || max_prefill > (1 << 24)) return false;
     Layout L;
     L.units = batch * kv_heads;
     L.cap = budget + 1;
     L.rowb = head_dim * elem_size(kv_dtype);
     L.lstride = round4(L.cap);
-    // every CTA range yields one item plus one more per unit boundary it crosses
-    L.max_items = kMaxCtas + L.units;
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes); return r; };
     L.status = take(256);
@@ -54,9 +57,19 @@ bool make_layout(int layers, int batch, int q_heads, int kv_heads, int head_dim,
     L.stage_k = take((size_t)batch * kv_heads * head_dim * 4);
     L.stage_v = take((size_t)batch * kv_heads * head_dim * 4);
     L.stage_out = take((size_t)batch * q_heads * head_dim * 4);
-    L.layer0 = o;
-    o = 0;
+    L.scratch0 = o;
     const size_t U = (size_t)L.units, C = (size_t)L.cap;
+    o = 0;
+    L.so.logit = take((size_t)batch * q_heads * L.lstride * 4);
+    L.so.part_o = take(U * kMaxParts * G * head_dim * 4);
+    L.so.part_ml = take(U * kMaxParts * G * 2 * 4);
+    L.so.keys = take(U * C * 8);
+    L.so.list_a = take(U * C * 4);
+    L.so.list_b = take(U * C * 4);
+    L.so.end = o;
+    L.scratch_bytes = o;
+    L.layer0 = L.scratch0 + L.scratch_bytes;
+    o = 0;
     L.lo.Kp = take(U * max_prefill * L.rowb);
     L.lo.Vp = take(U * max_prefill * L.rowb);
     L.lo.Kd = take(U * C * L.rowb);
@@ -64,24 +77,20 @@ bool make_layout(int layers, int batch, int q_heads, int kv_heads, int head_dim,
     L.lo.score = take(U * L.lstride * 4);
     L.lo.pos = take(U * L.lstride * 4);
     L.lo.n_dec = take(U * 4);
-    L.lo.logit = take((size_t)batch * q_heads * L.lstride * 4);
     L.lo.abar = take(U * C * 4);
     L.lo.n_prev = take(U * 4);
     L.lo.ev_k = take(U * 4);
     L.lo.ev_pos = take(U * C * 4);
     L.lo.ev_score = take(U * C * 4);
-    L.lo.items = take((size_t)L.max_items * sizeof(Item));
-    L.lo.cta_item0 = take((size_t)(kMaxCtas + 1) * 4);
+    L.lo.cta_unit0 = take((size_t)kMaxCtas * 4);
+    L.lo.cta_head0 = take((size_t)kMaxCtas * 4);
+    L.lo.cta_headn = take((size_t)kMaxCtas * 4);
     L.lo.unit_lp = take(U * 4);
-    L.lo.unit_part0 = take(U * 4);
-    L.lo.unit_nparts = take(U * 4);
-    L.lo.part_o = take((size_t)L.max_items * G * head_dim * 4);
-    L.lo.part_ml = take((size_t)L.max_items * G * 2 * 4);
-    L.lo.ticket = take(U * 4);
+    L.lo.unit_next0 = take(U * 4);
+    L.lo.next = take(2 * U * 4);      // two copies each, alternating from launch to launch
+    L.lo.done = take(2 * U * 4);
+    L.lo.nslots = take(2 * U * 4);
     L.lo.unit_step = take(U * 4);
-    L.lo.keys = take(U * C * 8);
-    L.lo.list_a = take(U * C * 4);
-    L.lo.list_b = take(U * C * 4);
     L.lo.end = o;
     L.layer_bytes = o;
     L.total = L.layer0 + L.layer_bytes * (size_t)layers;
@@ -126,8 +135,8 @@ struct mkv_ctx {
     std::vector<char> prefilled;
     std::vector<char> stepped;   // a step has run on the layer since its prefill
     bool pdl;
-    std::vector<int> n_items;
     std::vector<int> n_ctas;
+    std::vector<int64_t> layer_launches;   // steps launched on a layer: its parity picks the counter copy
     std::vector<std::vector<int32_t>> lens;   // per layer, per sequence
     int64_t launches;
 };
@@ -136,32 +145,41 @@ namespace {
 
 LayerDev layer_dev(const mkv_ctx* c, int layer) {
     uint8_t* base = c->ws + c->lay.layer0 + c->lay.layer_bytes * (size_t)layer;
+    uint8_t* sb = c->ws + c->lay.scratch0;
     const LayerOff& o = c->lay.lo;
+    const ScratchOff& so = c->lay.so;
+    const size_t U = (size_t)c->lay.units;
+    const size_t cur = (size_t)(c->layer_launches[layer] & 1), idle = cur ^ 1;
     LayerDev d;
     d.Kp = base + o.Kp; d.Vp = base + o.Vp; d.Kd = base + o.Kd; d.Vd = base + o.Vd;
     d.score = (float*)(base + o.score);
     d.pos = (int32_t*)(base + o.pos);
     d.n_dec = (int32_t*)(base + o.n_dec);
-    d.logit = (float*)(base + o.logit);
+    d.logit = (float*)(sb + so.logit);
     d.abar = (c->flags & MKV_FLAG_RECORD_PROBS) ? (float*)(base + o.abar) : nullptr;
     d.n_prev = (int32_t*)(base + o.n_prev);
     d.ev_k = (int32_t*)(base + o.ev_k);
     d.ev_pos = (int32_t*)(base + o.ev_pos);
     d.ev_score = (float*)(base + o.ev_score);
-    d.items = (const Item*)(base + o.items);
-    d.cta_item0 = (const int32_t*)(base + o.cta_item0);
-    d.n_items = c->n_items[layer];
+    d.n_units = c->lay.units;
     d.n_ctas = c->n_ctas[layer];
+    d.cta_unit0 = (const int32_t*)(base + o.cta_unit0);
+    d.cta_head0 = (const int32_t*)(base + o.cta_head0);
+    d.cta_headn = (const int32_t*)(base + o.cta_headn);
     d.unit_lp = (const int32_t*)(base + o.unit_lp);
-    d.unit_part0 = (const int32_t*)(base + o.unit_part0);
-    d.unit_nparts = (const int32_t*)(base + o.unit_nparts);
-    d.part_o = (float*)(base + o.part_o);
-    d.part_ml = (float*)(base + o.part_ml);
-    d.ticket = (int32_t*)(base + o.ticket);
+    d.unit_next0 = (const int32_t*)(base + o.unit_next0);
+    d.next = (int32_t*)(base + o.next) + cur * U;
+    d.done = (int32_t*)(base + o.done) + cur * U;
+    d.nslots = (int32_t*)(base + o.nslots) + cur * U;
+    d.next_idle = (int32_t*)(base + o.next) + idle * U;
+    d.done_idle = (int32_t*)(base + o.done) + idle * U;
+    d.nslots_idle = (int32_t*)(base + o.nslots) + idle * U;
+    d.part_o = (float*)(sb + so.part_o);
+    d.part_ml = (float*)(sb + so.part_ml);
     d.unit_step = (int32_t*)(base + o.unit_step);
-    d.keys = (unsigned long long*)(base + o.keys);
-    d.list_a = (int32_t*)(base + o.list_a);
-    d.list_b = (int32_t*)(base + o.list_b);
+    d.keys = (unsigned long long*)(sb + so.keys);
+    d.list_a = (int32_t*)(sb + so.list_a);
+    d.list_b = (int32_t*)(sb + so.list_b);
     return d;
 }
 
@@ -189,6 +207,7 @@ mkv_status launch_step(mkv_ctx* c, int layer, const Params& p, cudaStream_t st) 
     cudaError_t e = c->use_mma ? launch_mma(p, st, overlap) : launch_simt(p, c->kv_dtype, st);
     if (e != cudaSuccess) return MKV_ERR_CUDA;
     c->launches += 1;
+    c->layer_launches[layer] += 1;
     c->stepped[layer] = 1;
     return MKV_OK;
 }
@@ -272,8 +291,8 @@ mkv_status mkv_create(int layers, int q_heads, int kv_heads, int head_dim, int b
     c->stepped.assign(layers, 0);
     c->pdl = true;
     if (const char* e = std::getenv("MKV_NO_OVERLAP")) c->pdl = std::atoi(e) == 0;
-    c->n_items.assign(layers, 0);
     c->n_ctas.assign(layers, 0);
+    c->layer_launches.assign(layers, 0);
     c->lens.assign(layers, std::vector<int32_t>(batch, 0));
     c->launches = 0;
     *out_ctx = c;
@@ -298,67 +317,53 @@ mkv_status mkv_prefill(mkv_ctx* c, int layer, const void* K, const void* V, cons
     const Layout& L = c->lay;
     const int U = L.units;
 
-    // Static work list.  A unit's rows are a sequence of 64-row tiles (prefill tiles, then
-    // the decode tiles of the budget's row range); all units' tiles laid end to end are cut
-    // into equally long contiguous ranges, one per CTA; a range that crosses a unit
-    // boundary splits into items.  Ranges are long enough to keep a unit's item count
-    // within kMaxParts.
+    // Start table.  A unit's rows are a sequence of 64-row tiles (prefill tiles, then decode
+    // tiles); the CTAs are spread over the units in proportion to the units' tile counts (a
+    // full decode pool assumed).  Each CTA owns kHeadTiles tiles outright at its place, if the
+    // unit has that many prefill tiles left to give (these can be fetched before the previous
+    // step has finished); everything else is handed out by the unit's counter, which
+    // therefore starts behind the reserved tiles.
     const int td = ceil_div(c->budget_max, kTileRows);
-    std::vector<int32_t> lp(U), part0(U), nparts(U, 0);
+    std::vector<int32_t> lp(U), next0(U, 0);
     std::vector<long long> tile_begin(U + 1, 0);
-    int max_unit_tiles = 1;
     for (int u = 0; u < U; ++u) {
         lp[u] = prefill_lens[u / c->kv_heads];
-        const int tu = ceil_div(lp[u], kTileRows) + td;
-        tile_begin[u + 1] = tile_begin[u] + tu;
-        max_unit_tiles = std::max(max_unit_tiles, tu);
+        tile_begin[u + 1] = tile_begin[u] + ceil_div(lp[u], kTileRows) + td;
     }
     const long long t_all = tile_begin[U];
-    long long per_cta = std::max<long long>(ceil_div(max_unit_tiles, kMaxParts / 2 - 4), (t_all + c->n_ctas_max - 1) / c->n_ctas_max);
-    const int n_ctas = (int)((t_all + per_cta - 1) / per_cta);
-    std::vector<Item> items;
-    std::vector<int32_t> cta_item0(n_ctas + 1, 0);
+    const int n_ctas = (int)std::max<long long>(1, std::min<long long>(c->n_ctas_max, t_all / 2));
+    std::vector<int32_t> cta_unit0(n_ctas), cta_head0(n_ctas, 0), cta_headn(n_ctas, 0);
     {
         int u = 0;
         for (int cta = 0; cta < n_ctas; ++cta) {
-            cta_item0[cta] = (int32_t)items.size();
-            long long t0 = t_all * cta / n_ctas;
-            const long long t1 = t_all * (cta + 1) / n_ctas;
-            while (t0 < t1) {
-                while (tile_begin[u + 1] <= t0) ++u;
-                const long long e = std::min(t1, tile_begin[u + 1]);
-                items.push_back(Item{u, (int32_t)(t0 - tile_begin[u]), (int32_t)(e - t0), 0});
-                nparts[u] += 1;
-                t0 = e;
+            const long long t0 = t_all * cta / n_ctas;
+            while (tile_begin[u + 1] <= t0) ++u;
+            cta_unit0[cta] = u;
+            if (next0[u] + kHeadTiles <= ceil_div(lp[u], kTileRows)) {
+                cta_head0[cta] = next0[u];
+                cta_headn[cta] = kHeadTiles;
+                next0[u] += kHeadTiles;
             }
         }
-        cta_item0[n_ctas] = (int32_t)items.size();
     }
-    // partial index = item index; a unit's items are consecutive because ranges are in order
-    {
-        std::vector<char> seen(U, 0);
-        for (size_t i = 0; i < items.size(); ++i)
-            if (!seen[items[i].unit]) { seen[items[i].unit] = 1; part0[items[i].unit] = (int32_t)i; }
-    }
-    for (int u = 0; u < U; ++u)
-        if (nparts[u] < 1 || nparts[u] > kMaxParts) return MKV_ERR_CAPACITY;
-    if ((int)items.size() > L.max_items || n_ctas > kMaxCtas) return MKV_ERR_CAPACITY;
-    c->n_items[layer] = (int)items.size();
     c->n_ctas[layer] = n_ctas;
     for (int b = 0; b < c->batch; ++b) c->lens[layer][b] = prefill_lens[b];
 
     uint8_t* base = c->ws + L.layer0 + L.layer_bytes * (size_t)layer;
     bool ok = true;
-    ok &= cudaMemcpyAsync(base + L.lo.items, items.data(), items.size() * sizeof(Item), cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(base + L.lo.cta_item0, cta_item0.data(), cta_item0.size() * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(base + L.lo.cta_unit0, cta_unit0.data(), (size_t)n_ctas * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(base + L.lo.cta_head0, cta_head0.data(), (size_t)n_ctas * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(base + L.lo.cta_headn, cta_headn.data(), (size_t)n_ctas * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok &= cudaMemcpyAsync(base + L.lo.unit_lp, lp.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(base + L.lo.unit_part0, part0.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(base + L.lo.unit_nparts, nparts.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(base + L.lo.unit_next0, next0.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(base + L.lo.next, next0.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(base + L.lo.next + (size_t)U * 4, next0.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemsetAsync(base + L.lo.done, 0, 2 * (size_t)U * 4, st) == cudaSuccess;
+    ok &= cudaMemsetAsync(base + L.lo.nslots, 0, 2 * (size_t)U * 4, st) == cudaSuccess;
     // empty decode pool, rewind counters
     ok &= cudaMemsetAsync(base + L.lo.n_dec, 0, U * 4, st) == cudaSuccess;
     ok &= cudaMemsetAsync(base + L.lo.n_prev, 0, U * 4, st) == cudaSuccess;
     ok &= cudaMemsetAsync(base + L.lo.ev_k, 0, U * 4, st) == cudaSuccess;
-    ok &= cudaMemsetAsync(base + L.lo.ticket, 0, U * 4, st) == cudaSuccess;
     ok &= cudaMemsetAsync(base + L.lo.unit_step, 0, U * 4, st) == cudaSuccess;
     if (!ok) return MKV_ERR_CUDA;
     // host vectors above are pageable: the runtime has staged them before returning

@@ -19,13 +19,19 @@
 // per-element shuffling on the way in.
 //
 // Work decomposition.  The rows of a unit form a sequence of 64-row tiles: the prefill
-// tiles, then the decode tiles (over the budget's row range).  All tiles of all units,
-// laid end to end, are cut into one contiguous, equally long range per CTA; where a
-// range crosses a unit boundary it splits into "items".  An item (unit, first tile,
-// tile count) carries one online-softmax state across its tiles and yields one partial
-// (m, l, O[G][d]).  Whoever delivers the last partial of a unit (an atomic ticket, never
-// a wait) runs that unit's tail: the fresh token, combine, normalised decode
-// probabilities, head mean, momentum update, selection, append/compaction.
+// tiles, then the decode tiles that hold rows.  Tiles are handed out per unit by an atomic
+// counter, a few at a time.  Every CTA starts at its own place (CTAs are spread over the
+// units in proportion to the units' tile counts, and each owns a few reserved tiles there,
+// which it can fetch before anything else is known), then keeps pulling chunks of its unit
+// and, when that unit is exhausted, moves on to the next unit that still has tiles.  Fast
+// SMs therefore drift into the territory of slow ones and all CTAs finish together.  A CTA
+// carries one online-softmax state per unit visit and delivers it as one partial
+// (m, l, O[G][d]) together with the number of tiles it covered; the delivery that
+// completes the unit's tile count (an atomic add, never a wait) runs that unit's tail:
+// the fresh token, combine, normalised decode probabilities, head mean, momentum update,
+// selection, append/compaction.  The counters exist twice and alternate from launch to
+// launch; a unit's tail rewinds the idle copy, so no counter is ever reset while a CTA may
+// still probe it.
 //
 // The fresh token of a step never travels through the streaming part: its logit, its
 // probability, its importance and its row store all happen in the tail, which knows the
@@ -39,19 +45,13 @@ namespace mkv {
 
 constexpr int kTileRows = 64;       // rows of one tile of the work decomposition
 constexpr int kMaxGroup = 8;        // G = q_heads / kv_heads the kernels are built for
-constexpr int kMaxParts = 64;       // partials per unit (CTA ranges grow to keep this)
-constexpr int kMaxCtas = 2048;      // persistent grid upper bound (sizes the partial scratch)
+constexpr int kMaxParts = 64;       // partials per unit (chunks grow to keep this)
+constexpr int kMaxCtas = 2048;      // persistent grid upper bound
+constexpr int kHeadTiles = 3;       // tiles a CTA owns outright at its starting place
 constexpr float kNegBig = -1.0e30f; // finite stand-in for -inf in running maxima
 
 enum : int { kModeDecode = 0, kModeAttendOnly = 1 };
 enum : int { kStatusOk = 0, kStatusTimeout = 7, kStatusDeviceCheck = 8 };
-
-struct Item {          // 16 bytes, read as one int4
-    int32_t unit;
-    int32_t tile0;     // first tile inside the unit's tile sequence (prefill tiles first)
-    int32_t ntiles;
-    int32_t pad;
-};
 
 struct LayerDev {
     uint8_t *Kp, *Vp, *Kd, *Vd;
@@ -64,16 +64,21 @@ struct LayerDev {
     int32_t* ev_k;     // [units] tokens evicted by the last step
     int32_t* ev_pos;   // [units][cap]
     float* ev_score;   // [units][cap]
-    const Item* items;          // all items, CTA-major
-    const int32_t* cta_item0;   // [n_ctas + 1] first item of every CTA
-    int32_t n_items;
-    int32_t n_ctas;             // CTAs the work list was cut for (= the grid)
+    int32_t n_units;
+    int32_t n_ctas;             // the grid
+    const int32_t* cta_unit0;   // [n_ctas] unit a CTA starts in
+    const int32_t* cta_head0;   // [n_ctas] first of its reserved tiles there
+    const int32_t* cta_headn;   // [n_ctas] number of reserved tiles (prefill tiles; may be 0)
     const int32_t* unit_lp;     // [units] prefill length
-    const int32_t* unit_part0;  // [units] first partial index of the unit
-    const int32_t* unit_nparts; // [units]
-    float* part_o;     // [n_items][G][d]
-    float* part_ml;    // [n_items][G][2]  (running max in log2 units, running sum)
-    int32_t* ticket;   // [units]
+    const int32_t* unit_next0;  // [units] tiles reserved in the unit = start value of its counter
+    int32_t* next;     // [units] tiles handed out so far (this launch's copy)
+    int32_t* done;     // [units] tiles delivered so far
+    int32_t* nslots;   // [units] partial slots taken so far
+    int32_t* next_idle;   // the other copies, rewound by the tails for the next launch
+    int32_t* done_idle;
+    int32_t* nslots_idle;
+    float* part_o;     // [units][kMaxParts][G][d]
+    float* part_ml;    // [units][kMaxParts][G][2]  (running max in log2 units, running sum)
     int32_t* unit_step;// [units] decode steps completed
     unsigned long long* keys;   // [units][cap] selection scratch
     int32_t* list_a;   // [units][cap] compaction scratch (holes)
@@ -113,6 +118,13 @@ __device__ inline float fast_exp2(float x) {
 __device__ inline void bar_sync(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
+
+// Tiles of a unit that hold rows (at least one, so that every unit is visited and its tail
+// runs even when it has nothing cached yet) and the chunk handed out per pull.
+__device__ inline int unit_tiles(int lp, int n_old) {
+    return max(1, (lp + kTileRows - 1) / kTileRows + (n_old + kTileRows - 1) / kTileRows);
+}
+__device__ inline int unit_chunk(int total) { return max(2, (total + kMaxParts - 9) / (kMaxParts - 8)); }
 
 // Optional per-CTA timestamps (diagnostic builds only: compile with -DMKV_TRACE).  Slot i of
 // CTA c is g_trace[c * 16 + i]; mkv_debug_trace() copies the array to the host.

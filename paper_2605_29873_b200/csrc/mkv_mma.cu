@@ -4,14 +4,15 @@
 // Decode attention at GQA group 4-7 is bound by streaming K and V from HBM once per KV
 // head; the kernel is built around that stream.  A CTA is three kinds of warps:
 //
-//   * one PRODUCER thread walks the CTA's items of the static work list (a contiguous,
-//     equally long range of 64-row tiles per CTA) and issues bulk asynchronous copies (the
+//   * one PRODUCER thread pulls chunks of 64-row tiles from per-unit atomic counters,
+//     starting at the CTA's own place and moving on to the next unit with tiles left when
+//     its unit is exhausted, and issues bulk asynchronous copies (the
 //     non-tensor TMA form, no multicast) of K and V tiles, 16 KB each, into a ring of
 //     shared-memory stages; completion is signalled on an mbarrier (complete_tx).  The
 //     cache rows are already chunk-permuted in HBM, so a straight copy lands a layout that
-//     ldmatrix reads without bank conflicts.  At the start of an item it also copies the
-//     unit's G query rows into one of two small query slots.  The producer runs ahead
-//     across item boundaries.
+//     ldmatrix reads without bank conflicts.  At the start of a unit visit it also copies
+//     the unit's G query rows into one of two small query slots.  The producer runs ahead
+//     across unit boundaries.
 //   * four CONSUMER warps each own 16 rows of a tile and never synchronise with one
 //     another.  S = Q K^T uses mma.sync m16n8k16 (bf16 in, fp32 accumulate) with the G
 //     query heads in the M dimension; its accumulator fragment is, register for register,
@@ -24,10 +25,10 @@
 //     hi + lo bf16 halves, so the rounding of P to bf16 does not reach `out`.
 //     Raw fp32 logits of decode-pool tokens are stored (4 bytes per head and token) for
 //     the tail, which needs the global log-sum-exp before it can normalise them (Eq. 4).
-//   * four TAIL warps.  At the end of an item the consumers drop their (m, l, O) into a
-//     ring stage borrowed from the producer and go straight on to the next item; the tail
-//     warps merge the four states into one partial in global memory, take the unit's
-//     ticket and, when it is the last one, run the unit's tail (fresh token, combine,
+//   * four TAIL warps.  At the end of a unit visit the consumers drop their (m, l, O) into a
+//     ring stage borrowed from the producer and go straight on to the next unit; the tail
+//     warps merge the four states into one partial in global memory, add the visit's tiles
+//     to the unit's count and, when that completes it, run the unit's tail (fresh token, combine,
 //     probabilities, momentum update, selection, append/compaction) while the stream
 //     continues.
 // Every wait is bounded: on expiry the kernel records MKV_ERR_TIMEOUT, every role drains
@@ -62,15 +63,17 @@ enum : int { kEntryTile = 0, kEntryExchange = 1, kEntryEnd = 2 };
 struct StageMeta {
     int kind;
     int unit;
-    int item;
     int seg;        // 0 prefill, 1 decode
     int row;        // slot of the tile's first row inside its pool (multiple of 64)
     int cnt;        // valid rows
-    int first;      // first entry of its item: reset the running state
+    int first;      // first entry of a unit visit: reset the running state
+    int slot;       // exchange entries: the visit's partial slot ...
+    int ntiles;     // ... the tiles it covered ...
+    int total;      // ... and the unit's tile count
     int pad;
 };
 
-struct ExchangeRef { int stage, unit, item, pad; };
+struct ExchangeRef { int stage, unit, slot, ntiles, total; };   // stage < 0: no more exchanges
 
 struct Control {
     unsigned long long full[kMaxStages];
@@ -121,7 +124,6 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool dec = (p.mode == kModeDecode);
     const int G = p.group;
-    const int item_begin = L.cta_item0[blockIdx.x], item_end = L.cta_item0[blockIdx.x + 1];
 
     if (tid == 0) {
         for (int s = 0; s < nst; ++s) {
@@ -146,115 +148,172 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
 
     if (warp == kConsumerWarps) {
         // ================================ producer =====================================
+        // Lane 0 issues copies and pulls chunks; all lanes help when a new unit must be found.
+        int stage = 0;
+        uint32_t phase = 0;
+        uint32_t issued = 0;       // bit s: a copy into stage s may still be in flight
+        uint32_t issued_par = 0;   // parity its full barrier completes with
+        bool ok = true;
+        // K and V are read exactly once per step: let them leave L2 first, so that the
+        // step's scratch (logits, partials) and the scores stay resident for the tails
+        const unsigned long long stream_policy = ptx::l2_policy_evict_first();
+        int qcount = 0;            // visits that had at least one tile (and therefore a query slot)
+        auto acquire = [&]() -> bool {
+            if (!wait_or_abort(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl)) {
+                if (!aborted(ctl)) note_timeout(p, ctl);
+                return false;
+            }
+            issued &= ~(1u << stage);
+            return true;
+        };
+        auto advance = [&]() { if (++stage == nst) { stage = 0; phase ^= 1u; } };
+        auto issue_tile = [&](int u, const TileRef& tr, int first) -> bool {
+            if (!acquire()) return false;
+            StageMeta& mt = ctl->meta[stage];
+            mt.kind = kEntryTile; mt.unit = u; mt.seg = tr.seg; mt.row = tr.row; mt.cnt = tr.cnt; mt.first = first;
+            const uint32_t fb = ptx::smem_u32(&ctl->full[stage]);
+            const uint32_t dstK = ptx::smem_u32(stages + (size_t)stage * kStageBytes);
+            const size_t off = ((size_t)u * (tr.seg == 0 ? p.max_prefill : p.cap) + tr.row) * kRowB;
+            const uint8_t* kb = (tr.seg == 0 ? L.Kp : L.Kd) + off;
+            const uint8_t* vb = (tr.seg == 0 ? L.Vp : L.Vd) + off;
+            const uint32_t bytes = (uint32_t)tr.cnt * kRowB;
+            ptx::mbar_arrive_expect_tx(fb, 2u * bytes);
+            ptx::bulk_g2s_hint(dstK, kb, bytes, fb, stream_policy);
+            ptx::bulk_g2s_hint(dstK + kTileBytes, vb, bytes, fb, stream_policy);
+            issued |= 1u << stage;
+            issued_par = (issued_par & ~(1u << stage)) | (phase << stage);
+            advance();
+            return true;
+        };
+        // the unit's G query rows, one padded row each, into the next query slot
+        auto issue_query = [&](int u) -> bool {
+            const int b = u / p.kv_heads, g = u - b * p.kv_heads;
+            const int qi = qcount & 1;
+            if (!wait_or_abort(ptx::smem_u32(&ctl->qempty[qi]), (uint32_t)(((qcount >> 1) & 1) ^ 1), ctl)) {
+                if (!aborted(ctl)) note_timeout(p, ctl);
+                return false;
+            }
+            const uint32_t qb = ptx::smem_u32(&ctl->qfull[qi]);
+            const uint8_t* qsrc = reinterpret_cast<const uint8_t*>(p.q) + ((size_t)b * p.q_heads + (size_t)g * G) * kRowB;
+            ptx::mbar_arrive_expect_tx(qb, (uint32_t)G * kRowB);
+            for (int h = 0; h < G; ++h)
+                ptx::bulk_g2s(ptx::smem_u32(qslots + (size_t)qi * kQSlotBytes + (size_t)h * kQRowB),
+                              qsrc + (size_t)h * kRowB, kRowB, qb);
+            ++qcount;
+            if (dec) {   // the tail will want the fresh token's rows: bring them into L2 now
+                const uint8_t* kn = reinterpret_cast<const uint8_t*>(p.k_new) + (size_t)u * kRowB;
+                const uint8_t* vn = reinterpret_cast<const uint8_t*>(p.v_new) + (size_t)u * kRowB;
+                ptx::prefetch_l2(kn); ptx::prefetch_l2(kn + 128);
+                ptx::prefetch_l2(vn); ptx::prefetch_l2(vn + 128);
+            }
+            return true;
+        };
+        const int U = L.n_units;
+        int u = L.cta_unit0[blockIdx.x];
+        int lp = L.unit_lp[u];
+        // state of the current unit visit (lane 0)
+        int sent = 0;              // tile entries sent
+        int mine = 0;              // tiles covered, empty ones included
+        int slot = -1;             // the visit's partial slot (taken with the first tile)
+        bool q_sent = false;
+        // Before the dependency wait only data no earlier kernel of the stream writes may be
+        // touched: the start table and the frozen prefill pool.  The CTA's reserved tiles (prefill
+        // tiles by construction) are therefore in flight while the previous step still runs.
+        int head_t = 0, head_end = 0;   // reserved tiles still to issue (lane 0)
         if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            uint32_t issued = 0;       // bit s: a copy into stage s may still be in flight
-            uint32_t issued_par = 0;   // parity its full barrier completes with
-            bool ok = true;
-            // K and V are read exactly once per step: let them leave L2 first, so that the
-            // step's scratch (logits, partials) and the scores stay resident for the tails
-            const unsigned long long stream_policy = ptx::l2_policy_evict_first();
-            int qcount = 0;            // items that had at least one tile (and therefore a query slot)
-            auto acquire = [&]() -> bool {
-                if (!wait_or_abort(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl)) {
-                    if (!aborted(ctl)) note_timeout(p, ctl);
-                    return false;
+            head_t = L.cta_head0[blockIdx.x];
+            head_end = head_t + L.cta_headn[blockIdx.x];
+            // no more than the ring holds: the consumers only start after the wait
+            for (int n = 0; head_t < head_end && n < nst && ok; ++n, ++head_t) {
+                ok = issue_tile(u, tile_ref(head_t, lp, 0), sent == 0);
+                if (ok) { if (sent == 0) MKV_TR(1); ++sent; ++mine; }
+            }
+        }
+        ptx::griddep_wait();
+        int n_old = min(L.n_dec[u], p.cap - (dec ? 1 : 0));
+        int total = unit_tiles(lp, n_old);
+        int chunk = unit_chunk(total);
+        if (lane == 0 && ok && head_end > L.cta_head0[blockIdx.x]) {
+            slot = atomicAdd(&L.nslots[u], 1);
+            ok = issue_query(u);
+            q_sent = true;
+            for (; head_t < head_end && ok; ++head_t) {
+                ok = issue_tile(u, tile_ref(head_t, lp, 0), sent == 0);
+                ++sent; ++mine;
+            }
+        }
+        int g = 0;                 // first tile of the chunk in hand
+        if (lane == 0) g = atomicAdd(&L.next[u], chunk);
+        for (;;) {
+            g = __shfl_sync(0xffffffffu, g, 0);
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            if (g < total) {
+                if (lane == 0) {
+                    const int g_next = atomicAdd(&L.next[u], chunk);   // in flight while this chunk is issued
+                    if (slot < 0) slot = atomicAdd(&L.nslots[u], 1);
+                    const int t_end = min(g + chunk, total);
+                    for (int t = g; t < t_end && ok; ++t) {
+                        const TileRef tr = tile_ref(t, lp, n_old);
+                        ++mine;
+                        if (tr.cnt == 0) continue;
+                        if (!q_sent) { ok = issue_query(u); q_sent = true; if (!ok) break; }
+                        ok = issue_tile(u, tr, sent == 0);
+                        ++sent;
+                    }
+                    g = g_next;
                 }
-                issued &= ~(1u << stage);
-                return true;
-            };
-            auto advance = [&]() { if (++stage == nst) { stage = 0; phase ^= 1u; } };
-            auto issue_tile = [&](int u, int it, const TileRef& tr, int first) -> bool {
-                if (!acquire()) return false;
-                StageMeta& mt = ctl->meta[stage];
-                mt.kind = kEntryTile; mt.unit = u; mt.item = it; mt.seg = tr.seg; mt.row = tr.row;
-                mt.cnt = tr.cnt; mt.first = first;
-                const uint32_t fb = ptx::smem_u32(&ctl->full[stage]);
-                const uint32_t dstK = ptx::smem_u32(stages + (size_t)stage * kStageBytes);
-                const size_t off = ((size_t)u * (tr.seg == 0 ? p.max_prefill : p.cap) + tr.row) * kRowB;
-                const uint8_t* kb = (tr.seg == 0 ? L.Kp : L.Kd) + off;
-                const uint8_t* vb = (tr.seg == 0 ? L.Vp : L.Vd) + off;
-                const uint32_t bytes = (uint32_t)tr.cnt * kRowB;
-                ptx::mbar_arrive_expect_tx(fb, 2u * bytes);
-                ptx::bulk_g2s_hint(dstK, kb, bytes, fb, stream_policy);
-                ptx::bulk_g2s_hint(dstK + kTileBytes, vb, bytes, fb, stream_policy);
-                issued |= 1u << stage;
-                issued_par = (issued_par & ~(1u << stage)) | (phase << stage);
-                advance();
-                return true;
-            };
-            // the unit's G query rows, one padded row each, into the next query slot
-            auto issue_query = [&](int u) -> bool {
-                const int b = u / p.kv_heads, g = u - b * p.kv_heads;
-                const int qi = qcount & 1;
-                if (!wait_or_abort(ptx::smem_u32(&ctl->qempty[qi]), (uint32_t)(((qcount >> 1) & 1) ^ 1), ctl)) {
-                    if (!aborted(ctl)) note_timeout(p, ctl);
-                    return false;
+                continue;
+            }
+            // The unit has no tiles left to hand out: deliver this visit ...
+            if (lane == 0 && mine > 0) {
+                if ((ok = acquire())) {
+                    StageMeta& mt = ctl->meta[stage];
+                    mt.kind = kEntryExchange; mt.unit = u; mt.seg = 0; mt.row = 0; mt.cnt = 0; mt.first = (sent == 0);
+                    mt.slot = slot; mt.ntiles = mine; mt.total = total;
+                    ptx::mbar_arrive(ptx::smem_u32(&ctl->full[stage]));
+                    advance();
                 }
-                const uint32_t qb = ptx::smem_u32(&ctl->qfull[qi]);
-                const uint8_t* qsrc = reinterpret_cast<const uint8_t*>(p.q) + ((size_t)b * p.q_heads + (size_t)g * G) * kRowB;
-                ptx::mbar_arrive_expect_tx(qb, (uint32_t)G * kRowB);
-                for (int h = 0; h < G; ++h)
-                    ptx::bulk_g2s(ptx::smem_u32(qslots + (size_t)qi * kQSlotBytes + (size_t)h * kQRowB),
-                                  qsrc + (size_t)h * kRowB, kRowB, qb);
-                ++qcount;
-                if (dec) {   // the tail will want the fresh token's rows: bring them into L2 now
-                    const uint8_t* kn = reinterpret_cast<const uint8_t*>(p.k_new) + (size_t)u * kRowB;
-                    const uint8_t* vn = reinterpret_cast<const uint8_t*>(p.v_new) + (size_t)u * kRowB;
-                    ptx::prefetch_l2(kn); ptx::prefetch_l2(kn + 128);
-                    ptx::prefetch_l2(vn); ptx::prefetch_l2(vn + 128);
+                sent = 0; mine = 0; slot = -1; q_sent = false;
+            }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            // ... and look for the next unit (cyclically after this one) that still has some.
+            int found = -1;
+            for (int base = 1; base < U && found < 0; base += 32) {
+                const int k = base + lane;
+                int lpc = 0, ndc = 0;
+                bool has = false;
+                if (k < U) {
+                    const int cand = (u + k) % U;
+                    lpc = L.unit_lp[cand];
+                    ndc = min(L.n_dec[cand], p.cap - (dec ? 1 : 0));
+                    has = __ldcg(&L.next[cand]) < unit_tiles(lpc, ndc);
                 }
-                return true;
-            };
-            // Before the dependency wait: only data no earlier kernel of the stream writes may be
-            // touched -- the work list and the frozen prefill pool.  So the first item's leading
-            // prefill tiles are already in flight while the previous step finishes its tails.
-            int pre = 0;
-            if (item_begin < item_end) {
-                const int4 v = __ldg(reinterpret_cast<const int4*>(&L.items[item_begin]));
-                const int lp = L.unit_lp[v.x];
-                const int tp = (lp + kTileRows - 1) / kTileRows;
-                const int t_end = min(v.y + v.z, tp);
-                for (int t = v.y; t < t_end && pre < nst && ok; ++t) {
-                    const TileRef tr = tile_ref(t, lp, 0);
-                    ok = issue_tile(v.x, item_begin, tr, pre == 0);
-                    if (ok) { if (pre == 0) MKV_TR(1); ++pre; }
+                const unsigned ballot = __ballot_sync(0xffffffffu, has);
+                if (ballot) {
+                    const int src = __ffs(ballot) - 1;
+                    found = (u + base + src) % U;
+                    lp = __shfl_sync(0xffffffffu, lpc, src);
+                    n_old = __shfl_sync(0xffffffffu, ndc, src);
                 }
             }
-            ptx::griddep_wait();
-            for (int it = item_begin; it < item_end && ok; ++it) {
-                const int4 v = __ldg(reinterpret_cast<const int4*>(&L.items[it]));
-                const int u = v.x, tile0 = v.y, ntiles = v.z;
-                const int lp = L.unit_lp[u];
-                const int n_old = min(L.n_dec[u], p.cap - (dec ? 1 : 0));
-                int first = 1, t = tile0;
-                if (it == item_begin && pre > 0) { first = 0; t = tile0 + pre; }   // issued before the wait
-                // a non-empty first tile means the item has rows (empty decode tiles only trail)
-                if (tile_ref(tile0, lp, n_old).cnt > 0 && !(ok = issue_query(u))) break;
-                for (; t < tile0 + ntiles; ++t) {
-                    const TileRef tr = tile_ref(t, lp, n_old);
-                    if (tr.cnt == 0) continue;
-                    if (!(ok = issue_tile(u, it, tr, first))) break;
-                    first = 0;
-                }
-                if (!ok) break;
-                // the item's exchange entry: the consumers hand their state to the tail warps
-                if (!(ok = acquire())) break;
-                StageMeta& mt = ctl->meta[stage];
-                mt.kind = kEntryExchange; mt.unit = u; mt.item = it; mt.seg = 0; mt.row = 0; mt.cnt = 0; mt.first = first;
-                ptx::mbar_arrive(ptx::smem_u32(&ctl->full[stage]));
-                advance();
-            }
+            if (found < 0) break;
+            u = found;
+            total = unit_tiles(lp, n_old);
+            chunk = unit_chunk(total);
+            if (lane == 0) g = atomicAdd(&L.next[u], chunk);
+        }
+        if (lane == 0) {
             if (ok && acquire()) {
                 ctl->meta[stage].kind = kEntryEnd;
                 ptx::mbar_arrive(ptx::smem_u32(&ctl->full[stage]));
             } else {
                 // abort: leave only after every copy this thread issued has landed
-                for (int s = 0; s < nst; ++s)
-                    if (issued & (1u << s))
-                        wait_or_abort(ptx::smem_u32(&ctl->full[s]), (issued_par >> s) & 1u, ctl) ||
-                            ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->full[s]), (issued_par >> s) & 1u, kWaitNs);
+                for (int s2 = 0; s2 < nst; ++s2)
+                    if (issued & (1u << s2))
+                        wait_or_abort(ptx::smem_u32(&ctl->full[s2]), (issued_par >> s2) & 1u, ctl) ||
+                            ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->full[s2]), (issued_par >> s2) & 1u, kWaitNs);
             }
         }
         __syncwarp();
@@ -282,7 +341,14 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             }
             const StageMeta mt = ctl->meta[stage];
             if (warp == 0 && lane == 0 && xcount == 0 && mt.first) MKV_TR(2);
-            if (mt.kind == kEntryEnd) { if (warp == 0 && lane == 0) MKV_TR(3); break; }
+            if (mt.kind == kEntryEnd) {
+                if (warp == 0 && lane == 0) MKV_TR(3);
+                const int xs = xcount % nst;           // tells the tail warps that nothing follows
+                if (warp == 0 && lane == 0) ctl->xq[xs].stage = -1;
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->xfull[xs]));
+                break;
+            }
             uint8_t* const sK = stages + (size_t)stage * kStageBytes;
             uint8_t* const sV = sK + kTileBytes;
             if (mt.first) {
@@ -401,7 +467,8 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
                     ++qcount;
                 }
                 const int xs = xcount % nst;
-                if (warp == 0 && lane == 0) { ctl->xq[xs].stage = stage; ctl->xq[xs].unit = mt.unit; ctl->xq[xs].item = mt.item; }
+                if (warp == 0 && lane == 0) { ctl->xq[xs].stage = stage; ctl->xq[xs].unit = mt.unit; ctl->xq[xs].slot = mt.slot;
+                                             ctl->xq[xs].ntiles = mt.ntiles; ctl->xq[xs].total = mt.total; }
                 ptx::fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->xfull[xs]));
@@ -413,8 +480,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         // ================================ tail warps ===================================
         ptx::griddep_wait();
         const int tt = tid - kTailTid0;
-        const int n_mine = item_end - item_begin;
-        for (int x = 0; x < n_mine; ++x) {
+        for (int x = 0;; ++x) {
             const int xs = x % nst;
             if (tt == 0) {
                 const bool got = wait_or_abort(ptx::smem_u32(&ctl->xfull[xs]), (uint32_t)((x / nst) & 1), ctl);
@@ -424,11 +490,15 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             bar_sync(1, kTailThreads);
             if (!ctl->wait_ok) break;
             const ExchangeRef ref = ctl->xq[xs];
+            if (ref.stage < 0) break;
             const int u = ref.unit;
+            if (ref.slot < 0 || ref.slot >= kMaxParts) {     // cannot happen: chunks are sized to prevent it
+                if (tt == 0) atomicCAS(p.status, kStatusOk, kStatusDeviceCheck);
+            }
             const float* xo = reinterpret_cast<const float*>(stages + (size_t)ref.stage * kStageBytes);
             const float* xm = xo + kConsumerWarps * kMaxGroup * kXoStride;
             const float* xl = xm + kConsumerWarps * kMaxGroup;
-            const size_t part = (size_t)ref.item;
+            const size_t part = (size_t)u * kMaxParts + (size_t)min(max(ref.slot, 0), kMaxParts - 1);
             for (int idx = tt; idx < G * 128; idx += kTailThreads) {
                 const int h = idx >> 7, col = idx & 127;
                 float M = xm[h];
@@ -452,7 +522,8 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             bar_sync(1, kTailThreads);
             // the borrowed stage goes back to the producer
             if ((tt & 31) == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->empty[ref.stage]));
-            if (tt == 0) ctl->last_flag = (atomicAdd(&L.ticket[u], 1) == L.unit_nparts[u] - 1);
+            // the delivery that completes the unit's tile count runs its tail
+            if (tt == 0) ctl->last_flag = (atomicAdd(&L.done[u], ref.ntiles) + ref.ntiles == ref.total);
             bar_sync(1, kTailThreads);
             if (tt == 0) MKV_TR(4);
             if (ctl->last_flag) {

@@ -2,13 +2,14 @@
 // accepts.  It is the path for fp32 caches (where tensor cores would cost precision) and
 // the second, independent GPU implementation the tensor-core kernel is checked against.
 //
-// Persistent CTAs of four warps walk their items of the work list.  A warp owns whole
+// Persistent CTAs of four warps pull chunks of tiles from the per-unit counters, starting at
+// their own place and moving on to the next unit with tiles left.  A warp owns whole
 // cache rows: lane l holds head_dim/32 consecutive elements of the row, so a row is one
 // coalesced 128/256/512-byte access; the G query heads of the KV group share every K and V
 // row (GQA).  Per row: G dot products (Eq. 2 logits, already in log2 units), a butterfly
-// warp reduction, an online-softmax update of (m, l, O).  At the end of an item the warps
-// are merged in shared memory, the CTA writes one partial and takes the unit's ticket; the
-// last ticket holder runs the unit's tail.
+// warp reduction, an online-softmax update of (m, l, O).  At the end of a unit visit the warps
+// are merged in shared memory and the CTA writes one partial with its tile count; the
+// delivery that completes the unit runs its tail.
 #include "mkv_launch.h"
 #include "mkv_tail.cuh"
 
@@ -52,11 +53,13 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
     const LayerDev& L = p.L;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool dec = (p.mode == kModeDecode);
-    const int item_end = L.cta_item0[blockIdx.x + 1];
+    const int U = L.n_units;
+    __shared__ int s_g, s_u;
 
-    for (int it = L.cta_item0[blockIdx.x]; it < item_end; ++it) {
-        const int4 it4 = *reinterpret_cast<const int4*>(&L.items[it]);
-        const int u = it4.x, tile0 = it4.y, ntiles = it4.z;
+    int u = L.cta_unit0[blockIdx.x];
+    int head = L.cta_head0[blockIdx.x], headn = L.cta_headn[blockIdx.x];   // reserved tiles, first visit only
+    for (;;) {
+        // ---- one visit of unit u: pull chunks until the unit has none left -------------------
         const int b = u / p.kv_heads, g = u - b * p.kv_heads;
         const int lp = L.unit_lp[u];
         int n_old = L.n_dec[u];
@@ -64,7 +67,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
             if (tid == 0) atomicCAS(p.status, kStatusOk, kStatusDeviceCheck);
             n_old = p.cap - (dec ? 1 : 0);
         }
-
+        const int total = unit_tiles(lp, n_old), chunk = unit_chunk(total);
         float qf[G][EPL];
         {
             const T* qp = reinterpret_cast<const T*>(p.q) + ((size_t)b * p.q_heads + (size_t)g * G) * D + lane * EPL;
@@ -81,84 +84,112 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
             for (int e = 0; e < EPL; ++e) o[h][e] = 0.f;
         }
         float* lg = L.logit + ((size_t)b * p.q_heads + (size_t)g * G) * p.lstride;
-
-        for (int t = tile0; t < tile0 + ntiles; ++t) {
-            const TileRef tr = tile_ref(t, lp, n_old);
-            const uint8_t* kbase = (tr.seg == 0 ? L.Kp + (size_t)u * p.max_prefill * ROWB : L.Kd + (size_t)u * p.cap * ROWB);
-            const uint8_t* vbase = (tr.seg == 0 ? L.Vp + (size_t)u * p.max_prefill * ROWB : L.Vd + (size_t)u * p.cap * ROWB);
-            const bool store = dec && tr.seg == 1;
-            for (int r = tr.row + warp; r < tr.row + tr.cnt; r += kSimtWarps) {
-                float kf[EPL], vf[EPL];
-                const uint32_t off = swz((uint32_t)r, (uint32_t)(lane * BPL));
-                load_piece<T, EPL>(kbase + (size_t)r * ROWB + off, kf);
-                load_piece<T, EPL>(vbase + (size_t)r * ROWB + off, vf);
-                float s[G];
+        int mine = 0;
+        for (;;) {
+            int t0, t1;
+            if (headn > 0) { t0 = head; t1 = head + headn; headn = 0; }
+            else {
+                if (tid == 0) s_g = atomicAdd(&L.next[u], chunk);
+                __syncthreads();
+                t0 = s_g;
+                __syncthreads();
+                if (t0 >= total) break;
+                t1 = min(t0 + chunk, total);
+            }
+            mine += t1 - t0;
+            for (int t = t0; t < t1; ++t) {
+                const TileRef tr = tile_ref(t, lp, n_old);
+                const uint8_t* kbase = (tr.seg == 0 ? L.Kp + (size_t)u * p.max_prefill * ROWB : L.Kd + (size_t)u * p.cap * ROWB);
+                const uint8_t* vbase = (tr.seg == 0 ? L.Vp + (size_t)u * p.max_prefill * ROWB : L.Vd + (size_t)u * p.cap * ROWB);
+                const bool store = dec && tr.seg == 1;
+                for (int r = tr.row + warp; r < tr.row + tr.cnt; r += kSimtWarps) {
+                    float kf[EPL], vf[EPL];
+                    const uint32_t off = swz((uint32_t)r, (uint32_t)(lane * BPL));
+                    load_piece<T, EPL>(kbase + (size_t)r * ROWB + off, kf);
+                    load_piece<T, EPL>(vbase + (size_t)r * ROWB + off, vf);
+                    float sc[G];
 #pragma unroll
-                for (int h = 0; h < G; ++h) {
-                    float a = 0.f;
+                    for (int h = 0; h < G; ++h) {
+                        float a = 0.f;
 #pragma unroll
-                    for (int e = 0; e < EPL; ++e) a = fmaf(qf[h][e], kf[e], a);
-                    s[h] = a;
+                        for (int e = 0; e < EPL; ++e) a = fmaf(qf[h][e], kf[e], a);
+                        sc[h] = a;
+                    }
+#pragma unroll
+                    for (int off2 = 16; off2; off2 >>= 1)
+#pragma unroll
+                        for (int h = 0; h < G; ++h) sc[h] += __shfl_xor_sync(0xffffffffu, sc[h], off2);
+#pragma unroll
+                    for (int h = 0; h < G; ++h) {
+                        if (store && lane == h) lg[(size_t)h * p.lstride + r] = sc[h];
+                        const float mn = fmaxf(m[h], sc[h]);
+                        const float fs = fast_exp2(m[h] - mn);
+                        const float pr = fast_exp2(sc[h] - mn);
+                        l[h] = fmaf(l[h], fs, pr);
+#pragma unroll
+                        for (int e = 0; e < EPL; ++e) o[h][e] = fmaf(o[h][e], fs, pr * vf[e]);
+                        m[h] = mn;
+                    }
                 }
+            }
+        }
+        if (mine > 0) {
+            // merge the four warps, write the visit's partial into a fresh slot of the unit
+            if (tid == 0) s_g = atomicAdd(&L.nslots[u], 1);
+            if (lane == 0) {
 #pragma unroll
-                for (int off2 = 16; off2; off2 >>= 1)
+                for (int h = 0; h < G; ++h) { xm[warp][h] = m[h]; xl[warp][h] = l[h]; }
+            }
 #pragma unroll
-                    for (int h = 0; h < G; ++h) s[h] += __shfl_xor_sync(0xffffffffu, s[h], off2);
+            for (int h = 0; h < G; ++h)
 #pragma unroll
-                for (int h = 0; h < G; ++h) {
-                    if (store && lane == h) lg[(size_t)h * p.lstride + r] = s[h];
-                    const float mn = fmaxf(m[h], s[h]);
-                    const float sc = fast_exp2(m[h] - mn);
-                    const float pr = fast_exp2(s[h] - mn);
-                    l[h] = fmaf(l[h], sc, pr);
+                for (int e = 0; e < EPL; ++e) xo[warp][h][lane * EPL + e] = o[h][e];
+            __syncthreads();
+            if (s_g >= kMaxParts && tid == 0) atomicCAS(p.status, kStatusOk, kStatusDeviceCheck);
+            const size_t part = (size_t)u * kMaxParts + (size_t)min(s_g, kMaxParts - 1);
+            for (int idx = tid; idx < G * D; idx += kSimtThreads) {
+                const int h = idx / D, i = idx - h * D;
+                float M = xm[0][h];
 #pragma unroll
-                    for (int e = 0; e < EPL; ++e) o[h][e] = fmaf(o[h][e], sc, pr * vf[e]);
-                    m[h] = mn;
+                for (int w = 1; w < kSimtWarps; ++w) M = fmaxf(M, xm[w][h]);
+                float acc = 0.f, ls = 0.f;
+#pragma unroll
+                for (int w = 0; w < kSimtWarps; ++w) {
+                    const float fs = fast_exp2(xm[w][h] - M);
+                    acc = fmaf(xo[w][h][i], fs, acc);
+                    ls = fmaf(xl[w][h], fs, ls);
+                }
+                L.part_o[part * G * D + idx] = acc;
+                if (i == 0) {
+                    L.part_ml[(part * G + h) * 2] = M;
+                    L.part_ml[(part * G + h) * 2 + 1] = ls;
                 }
             }
-        }
-
-        // merge the four warps, write the partial
-        if (lane == 0) {
-#pragma unroll
-            for (int h = 0; h < G; ++h) { xm[warp][h] = m[h]; xl[warp][h] = l[h]; }
-        }
-#pragma unroll
-        for (int h = 0; h < G; ++h)
-#pragma unroll
-            for (int e = 0; e < EPL; ++e) xo[warp][h][lane * EPL + e] = o[h][e];
-        __syncthreads();
-        const size_t part = (size_t)it;
-        for (int idx = tid; idx < G * D; idx += kSimtThreads) {
-            const int h = idx / D, i = idx - h * D;
-            float M = xm[0][h];
-#pragma unroll
-            for (int w = 1; w < kSimtWarps; ++w) M = fmaxf(M, xm[w][h]);
-            float acc = 0.f, ls = 0.f;
-#pragma unroll
-            for (int w = 0; w < kSimtWarps; ++w) {
-                const float sc = fast_exp2(xm[w][h] - M);
-                acc = fmaf(xo[w][h][i], sc, acc);
-                ls = fmaf(xl[w][h], sc, ls);
-            }
-            L.part_o[part * G * D + idx] = acc;
-            if (i == 0) {
-                L.part_ml[(part * G + h) * 2] = M;
-                L.part_ml[(part * G + h) * 2 + 1] = ls;
-            }
-        }
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) {
-            const int prev = atomicAdd(&L.ticket[u], 1);
-            s_last = (prev == L.unit_nparts[u] - 1);
-        }
-        __syncthreads();
-        if (s_last) {
             __threadfence();
-            unit_tail<T, kSimtThreads, 1, (G <= 4 ? 4 : 8)>(p, load_tail_job(L, u), tsm, tid);
+            __syncthreads();
+            // the delivery that completes the unit's tile count runs its tail
+            if (tid == 0) s_last = (atomicAdd(&L.done[u], mine) + mine == total);
+            __syncthreads();
+            if (s_last) {
+                __threadfence();
+                unit_tail<T, kSimtThreads, 1, (G <= 4 ? 4 : 8)>(p, load_tail_job(L, u), tsm, tid);
+            }
+            __syncthreads();
+        }
+        // ---- next unit (cyclically after this one) that still has tiles to hand out -----------
+        if (tid == 0) {
+            int found = -1;
+            for (int k = 1; k < U; ++k) {
+                const int cand = (u + k) % U;
+                const int nd = min(L.n_dec[cand], p.cap - (dec ? 1 : 0));
+                if (__ldcg(&L.next[cand]) < unit_tiles(L.unit_lp[cand], nd)) { found = cand; break; }
+            }
+            s_u = found;
         }
         __syncthreads();
+        u = s_u;
+        __syncthreads();
+        if (u < 0) break;
     }
 }
 

@@ -87,8 +87,15 @@ struct TailJob { int u, P, part0, n_dec, t; };
 
 __device__ inline TailJob load_tail_job(const LayerDev& L, int u) {
     TailJob j;
-    j.u = u; j.P = L.unit_nparts[u]; j.part0 = L.unit_part0[u]; j.n_dec = L.n_dec[u]; j.t = L.unit_step[u];
+    j.u = u; j.P = min(__ldcg(&L.nslots[u]), kMaxParts); j.part0 = u * kMaxParts; j.n_dec = L.n_dec[u]; j.t = L.unit_step[u];
     return j;
+}
+
+// The unit is complete: prepare the idle copy of its counters for the next launch.
+__device__ inline void rewind_unit(const LayerDev& L, int u) {
+    L.next_idle[u] = L.unit_next0[u];
+    L.done_idle[u] = 0;
+    L.nslots_idle[u] = 0;
 }
 
 __device__ inline void store_out4(const Params& p, size_t idx, float4 v) {
@@ -279,7 +286,7 @@ __device__ void unit_tail(const Params& p, const TailJob& job, TailSmem<NT>& sm,
     if (!dec) {
         finish_out();
         if (tid == 0) MKV_TR(11);
-        if (tid == 0) L.ticket[u] = 0;
+        if (tid == 0) rewind_unit(L, u);
         return;
     }
     if (tid == 0) MKV_TR(11);
@@ -354,7 +361,7 @@ __device__ void unit_tail(const Params& p, const TailJob& job, TailSmem<NT>& sm,
         if (warp == (NW > 1 ? 1 : 0)) store_row_swizzled(L.Vd, ubase, rowb, vnew, n_old, lane);
         if (tid == NT - 1) { score[n_old] = ab_new; pos[n_old] = t; keys[n_old] = key_new; }
         if (k == 0) {
-            if (tid == 0) L.ticket[u] = 0;
+            if (tid == 0) rewind_unit(L, u);
             return;
         }
     }
@@ -385,7 +392,7 @@ __device__ void unit_tail(const Params& p, const TailJob& job, TailSmem<NT>& sm,
             if (warp == (NW > 1 ? 1 : 0)) store_row_swizzled(L.Vd, ubase, rowb, vnew, e, lane);
             if (tid == NT - 1) { score[e] = ab_new; pos[e] = t; }
         }
-        if (tid == 0) L.ticket[u] = 0;
+        if (tid == 0) rewind_unit(L, u);
         return;
     }
 
@@ -461,7 +468,7 @@ __device__ void unit_tail(const Params& p, const TailJob& job, TailSmem<NT>& sm,
             if (lane == 0) { score[dst] = score[src]; pos[dst] = pos[src]; }
         }
     }
-    if (tid == 0) L.ticket[u] = 0;
+    if (tid == 0) rewind_unit(L, u);
 }
 
 }  // namespace mkv
