@@ -2,7 +2,7 @@
 // path of the Llama-3.1-8B- and Qwen2.5-7B-shaped workloads.
 //
 // Decode attention at GQA group 4-7 is bound by streaming K and V from HBM once per KV
-// head; the kernel is built around that stream.  A CTA is three kinds of warps:
+// head; the kernel is built around that stream.  A CTA is four kinds of warps:
 //
 //   * one PRODUCER thread pulls chunks of 64-row tiles from per-unit atomic counters,
 //     starting at the CTA's own place and moving on to the next unit with tiles left when
@@ -25,12 +25,14 @@
 //     hi + lo bf16 halves, so the rounding of P to bf16 does not reach `out`.
 //     Raw fp32 logits of decode-pool tokens are stored (4 bytes per head and token) for
 //     the tail, which needs the global log-sum-exp before it can normalise them (Eq. 4).
-//   * four TAIL warps.  At the end of a unit visit the consumers drop their (m, l, O) into a
-//     ring stage borrowed from the producer and go straight on to the next unit; the tail
-//     warps merge the four states into one partial in global memory, add the visit's tiles
-//     to the unit's count and, when that completes it, run the unit's tail (fresh token, combine,
-//     probabilities, momentum update, selection, append/compaction) while the stream
-//     continues.
+//   * one MERGE warp.  At the end of a unit visit the consumers drop their (m, l, O) into a
+//     ring stage borrowed from the producer and go straight on to the next unit; the merge
+//     warp folds the four states into one partial in global memory, returns the stage, adds
+//     the visit's tiles to the unit's count and, when that completes it, publishes the unit
+//     in the layer's queue of due tails.
+//   * four TAIL warps, which claim entries of that queue (one group per entry, across all
+//     CTAs) and run the unit tails (fresh token, combine, probabilities, momentum update,
+//     selection, append/compaction) while the stream continues.
 // Every wait is bounded: on expiry the kernel records MKV_ERR_TIMEOUT, every role drains
 // (the producer waits, bounded again, for its copies in flight) and the CTA returns.
 #include <cstdlib>
@@ -50,10 +52,11 @@ constexpr int kQSlotBytes = kMaxGroup * kQRowB;           // query rows of one u
 constexpr int kQSlots = 2;
 constexpr int kConsumerWarps = 4;
 constexpr int kTailWarps = 4;
-constexpr int kConsumers = kConsumerWarps * 32;
 constexpr int kTailThreads = kTailWarps * 32;
-constexpr int kTailTid0 = kConsumers + 32;                // first thread of the tail group
-constexpr int kThreads = kConsumers + 32 + kTailThreads;
+constexpr int kProducerWarp = kConsumerWarps;             // warp 4
+constexpr int kMergeWarp = kConsumerWarps + 1;            // warp 5
+constexpr int kTailTid0 = (kMergeWarp + 1) * 32;          // first thread of the tail group
+constexpr int kThreads = kTailTid0 + kTailThreads;
 constexpr int kMaxStages = 8;
 constexpr int kXoStride = 132;                            // floats per head row of the exchange
 constexpr unsigned long long kWaitNs = 2000000000ull;     // 2 s
@@ -84,8 +87,8 @@ struct Control {
     StageMeta meta[kMaxStages];
     ExchangeRef xq[kMaxStages];
     int abort_flag;
-    int last_flag;
-    int wait_ok;
+    int tail_entry;    // queue index the tail warps hold, or -1
+    int tail_unit;
 };
 
 constexpr size_t smem_bytes(int nst) {
@@ -136,8 +139,8 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             ptx::mbar_init(ptx::smem_u32(&ctl->qempty[s]), kConsumerWarps);
         }
         ctl->abort_flag = 0;
-        ctl->last_flag = 0;
-        ctl->wait_ok = 1;
+        ctl->tail_entry = -1;
+        ctl->tail_unit = -1;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async();
     }
@@ -146,7 +149,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
     // The next kernel of the stream may start as soon as SMs free up; it does its own waiting.
     ptx::griddep_launch_dependents();
 
-    if (warp == kConsumerWarps) {
+    if (warp == kProducerWarp) {
         // ================================ producer =====================================
         // Lane 0 issues copies and pulls chunks; all lanes help when a new unit must be found.
         int stage = 0;
@@ -476,65 +479,107 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             }
             if (++stage == nst) { stage = 0; phase ^= 1u; }
         }
-    } else {
-        // ================================ tail warps ===================================
+    } else if (warp == kMergeWarp) {
+        // ================================ merge warp ===================================
+        // Folds the four consumer states of a unit visit into one partial in global memory,
+        // gives the borrowed stage back, adds the visit's tiles to the unit's count and, when
+        // that completes the unit, publishes the unit in the layer's queue of due tails.
         ptx::griddep_wait();
-        const int tt = tid - kTailTid0;
         for (int x = 0;; ++x) {
             const int xs = x % nst;
-            if (tt == 0) {
-                const bool got = wait_or_abort(ptx::smem_u32(&ctl->xfull[xs]), (uint32_t)((x / nst) & 1), ctl);
-                if (!got && !aborted(ctl)) note_timeout(p, ctl);
-                ctl->wait_ok = got ? 1 : 0;
+            if (!wait_or_abort(ptx::smem_u32(&ctl->xfull[xs]), (uint32_t)((x / nst) & 1), ctl)) {
+                if (lane == 0 && !aborted(ctl)) note_timeout(p, ctl);
+                break;
             }
-            bar_sync(1, kTailThreads);
-            if (!ctl->wait_ok) break;
             const ExchangeRef ref = ctl->xq[xs];
             if (ref.stage < 0) break;
             const int u = ref.unit;
             if (ref.slot < 0 || ref.slot >= kMaxParts) {     // cannot happen: chunks are sized to prevent it
-                if (tt == 0) atomicCAS(p.status, kStatusOk, kStatusDeviceCheck);
+                if (lane == 0) atomicCAS(p.status, kStatusOk, kStatusDeviceCheck);
             }
             const float* xo = reinterpret_cast<const float*>(stages + (size_t)ref.stage * kStageBytes);
             const float* xm = xo + kConsumerWarps * kMaxGroup * kXoStride;
             const float* xl = xm + kConsumerWarps * kMaxGroup;
             const size_t part = (size_t)u * kMaxParts + (size_t)min(max(ref.slot, 0), kMaxParts - 1);
-            for (int idx = tt; idx < G * 128; idx += kTailThreads) {
-                const int h = idx >> 7, col = idx & 127;
+            for (int h = 0; h < G; ++h) {
                 float M = xm[h];
 #pragma unroll
                 for (int w = 1; w < kConsumerWarps; ++w) M = fmaxf(M, xm[w * kMaxGroup + h]);
-                float acc = 0.f, ls = 0.f;
+                float wsc[kConsumerWarps];
+                float ls = 0.f;
 #pragma unroll
                 for (int w = 0; w < kConsumerWarps; ++w) {
-                    const float wsc = fast_exp2(xm[w * kMaxGroup + h] - M);
-                    acc = fmaf(xo[(size_t)(w * kMaxGroup + h) * kXoStride + col], wsc, acc);
-                    ls = fmaf(xl[w * kMaxGroup + h], wsc, ls);
+                    wsc[w] = fast_exp2(xm[w * kMaxGroup + h] - M);
+                    ls = fmaf(xl[w * kMaxGroup + h], wsc[w], ls);
                 }
-                L.part_o[(part * G + h) * 128 + col] = acc;
-                if (col == 0) {
-                    L.part_ml[(part * G + h) * 2] = M;
-                    L.part_ml[(part * G + h) * 2 + 1] = ls;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) {
+                    const float4 v = *reinterpret_cast<const float4*>(xo + (size_t)(w * kMaxGroup + h) * kXoStride + 4 * lane);
+                    acc.x = fmaf(v.x, wsc[w], acc.x); acc.y = fmaf(v.y, wsc[w], acc.y);
+                    acc.z = fmaf(v.z, wsc[w], acc.z); acc.w = fmaf(v.w, wsc[w], acc.w);
                 }
+                *reinterpret_cast<float4*>(&L.part_o[(part * G + h) * 128 + 4 * lane]) = acc;
+                if (lane == 0) *reinterpret_cast<float2*>(&L.part_ml[(part * G + h) * 2]) = make_float2(M, ls);
             }
-            __threadfence();
+            __syncwarp();
             ptx::fence_proxy_async();
-            bar_sync(1, kTailThreads);
-            // the borrowed stage goes back to the producer
-            if ((tt & 31) == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->empty[ref.stage]));
-            // the delivery that completes the unit's tile count runs its tail
-            if (tt == 0) ctl->last_flag = (atomicAdd(&L.done[u], ref.ntiles) + ref.ntiles == ref.total);
-            bar_sync(1, kTailThreads);
-            if (tt == 0) MKV_TR(4);
-            if (ctl->last_flag) {
-                if (tt == 0) MKV_TR_ADD(6, 1);
-                __threadfence();
-                const TailJob job = load_tail_job(L, u);
-                if (G <= 4) unit_tail<__nv_bfloat16, kTailThreads, 1, 4>(p, job, *tsm, tt);
-                else unit_tail<__nv_bfloat16, kTailThreads, 1, 8>(p, job, *tsm, tt);
+            // the borrowed stage goes back to the producer (its empty barrier counts four arrivals)
+            if (lane < kConsumerWarps) ptx::mbar_arrive(ptx::smem_u32(&ctl->empty[ref.stage]));
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) {
+                MKV_TR(4);
+                // the delivery that completes the unit's tile count makes its tail due
+                if (atomicAdd(&L.done[u], ref.ntiles) + ref.ntiles == ref.total) {
+                    const int idx = atomicAdd(&L.tq_pub[0], 1);
+                    if (idx < L.n_units) {
+                        L.tq_unit[idx] = u;
+                        __threadfence();
+                        atomicExch(&L.tq_ready[idx], 1);
+                    } else {
+                        atomicCAS(p.status, kStatusOk, kStatusDeviceCheck);
+                    }
+                }
+            }
+        }
+    } else {
+        // ================================ tail warps ===================================
+        // Unit tails are served from one queue per layer: each tail group claims the next
+        // queue index and waits for that entry to be published, so every due tail finds an
+        // idle group of its own and no CTA ever has two to run.  Groups whose index lies
+        // beyond the number of units have nothing to wait for.
+        ptx::griddep_wait();
+        const int tt = tid - kTailTid0;
+        for (;;) {
+            if (tt == 0) {
+                int my = atomicAdd(&L.tq_claim[0], 1), unit = -1;
+                if (my < L.n_units) {
+                    const unsigned long long t0 = ptx::globaltimer_ns();
+                    for (;;) {
+                        if (*reinterpret_cast<volatile int*>(&L.tq_ready[my]) != 0) { __threadfence(); unit = __ldcg(&L.tq_unit[my]); break; }
+                        if (aborted(ctl)) break;
+                        if (ptx::globaltimer_ns() - t0 > kWaitNs) { note_timeout(p, ctl); break; }
+                        __nanosleep(200);
+                    }
+                }
+                ctl->tail_entry = unit >= 0 ? my : -1;
+                ctl->tail_unit = unit;
             }
             bar_sync(1, kTailThreads);
-            if (tt == 0) MKV_TR(5);
+            const int my = ctl->tail_entry, u = ctl->tail_unit;
+            bar_sync(1, kTailThreads);     // everyone has read them before thread 0 writes again
+            if (my < 0) break;
+            if (tt == 0) MKV_TR_ADD(6, 1);
+            const TailJob job = load_tail_job(L, u);
+            if (G <= 4) unit_tail<__nv_bfloat16, kTailThreads, 1, 4>(p, job, *tsm, tt);
+            else unit_tail<__nv_bfloat16, kTailThreads, 1, 8>(p, job, *tsm, tt);
+            // rewind the idle copy of the queue for the launch after next
+            if (tt == 0) {
+                L.tq_ready_idle[my] = 0;
+                if (my == 0) { L.tq_claim_idle[0] = 0; L.tq_pub_idle[0] = 0; }
+                MKV_TR(5);
+            }
         }
     }
 }
