@@ -23,7 +23,7 @@ inline int elem_size(int dt) { return dt == MKV_BF16 ? 2 : 4; }
 
 struct LayerOff {
     size_t Kp, Vp, Kd, Vd, score, pos, n_dec, abar, n_prev, ev_k, ev_pos, ev_score, cta_unit0, cta_head0,
-        cta_headn, unit_lp, unit_next0, next, done, nslots, tq_ctl, tq_ready, tq_unit, unit_step, end;
+        cta_headn, unit_lp, unit_next0, next, done, nslots, unit_step, end;
 };
 // Scratch that lives for one step only, shared by all layers of the context (calls on a
 // context are ordered on one stream, and a step touches it only after every earlier kernel
@@ -90,9 +90,6 @@ bool make_layout(int layers, int batch, int q_heads, int kv_heads, int head_dim,
     L.lo.next = take(2 * U * 4);      // two copies each, alternating from launch to launch
     L.lo.done = take(2 * U * 4);
     L.lo.nslots = take(2 * U * 4);
-    L.lo.tq_ctl = take(2 * 256);      // claim and publish counters, two copies
-    L.lo.tq_ready = take(2 * U * 4);
-    L.lo.tq_unit = take(2 * U * 4);
     L.lo.unit_step = take(U * 4);
     L.lo.end = o;
     L.layer_bytes = o;
@@ -177,13 +174,6 @@ LayerDev layer_dev(const mkv_ctx* c, int layer) {
     d.next_idle = (int32_t*)(base + o.next) + idle * U;
     d.done_idle = (int32_t*)(base + o.done) + idle * U;
     d.nslots_idle = (int32_t*)(base + o.nslots) + idle * U;
-    d.tq_claim = (int32_t*)(base + o.tq_ctl + cur * 256);
-    d.tq_pub = d.tq_claim + 32;
-    d.tq_ready = (int32_t*)(base + o.tq_ready) + cur * U;
-    d.tq_unit = (int32_t*)(base + o.tq_unit) + cur * U;
-    d.tq_claim_idle = (int32_t*)(base + o.tq_ctl + idle * 256);
-    d.tq_pub_idle = d.tq_claim_idle + 32;
-    d.tq_ready_idle = (int32_t*)(base + o.tq_ready) + idle * U;
     d.part_o = (float*)(sb + so.part_o);
     d.part_ml = (float*)(sb + so.part_ml);
     d.unit_step = (int32_t*)(base + o.unit_step);
@@ -370,8 +360,6 @@ mkv_status mkv_prefill(mkv_ctx* c, int layer, const void* K, const void* V, cons
     ok &= cudaMemcpyAsync(base + L.lo.next + (size_t)U * 4, next0.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok &= cudaMemsetAsync(base + L.lo.done, 0, 2 * (size_t)U * 4, st) == cudaSuccess;
     ok &= cudaMemsetAsync(base + L.lo.nslots, 0, 2 * (size_t)U * 4, st) == cudaSuccess;
-    ok &= cudaMemsetAsync(base + L.lo.tq_ctl, 0, 2 * 256, st) == cudaSuccess;
-    ok &= cudaMemsetAsync(base + L.lo.tq_ready, 0, 2 * (size_t)U * 4, st) == cudaSuccess;
     // empty decode pool, rewind counters
     ok &= cudaMemsetAsync(base + L.lo.n_dec, 0, U * 4, st) == cudaSuccess;
     ok &= cudaMemsetAsync(base + L.lo.n_prev, 0, U * 4, st) == cudaSuccess;

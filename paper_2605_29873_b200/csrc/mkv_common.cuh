@@ -77,14 +77,6 @@ struct LayerDev {
     int32_t* next_idle;   // the other copies, rewound by the tails for the next launch
     int32_t* done_idle;
     int32_t* nslots_idle;
-    // queue of due unit tails (tensor-core kernel): again two alternating copies
-    int32_t* tq_claim;    // [1] queue indices claimed by tail groups
-    int32_t* tq_pub;      // [1] queue indices published
-    int32_t* tq_ready;    // [units] entry published
-    int32_t* tq_unit;     // [units] the unit of an entry
-    int32_t* tq_claim_idle;
-    int32_t* tq_pub_idle;
-    int32_t* tq_ready_idle;
     float* part_o;     // [units][kMaxParts][G][d]
     float* part_ml;    // [units][kMaxParts][G][2]  (running max in log2 units, running sum)
     int32_t* unit_step;// [units] decode steps completed

@@ -28,11 +28,10 @@
 //   * one MERGE warp.  At the end of a unit visit the consumers drop their (m, l, O) into a
 //     ring stage borrowed from the producer and go straight on to the next unit; the merge
 //     warp folds the four states into one partial in global memory, returns the stage, adds
-//     the visit's tiles to the unit's count and, when that completes it, publishes the unit
-//     in the layer's queue of due tails.
-//   * four TAIL warps, which claim entries of that queue (one group per entry, across all
-//     CTAs) and run the unit tails (fresh token, combine, probabilities, momentum update,
-//     selection, append/compaction) while the stream continues.
+//     the visit's tiles to the unit's count.
+//   * four TAIL warps, which watch the counts of the units assigned to this CTA and run a
+//     unit's tail (fresh token, combine, probabilities, momentum update, selection,
+//     append/compaction) as soon as its count is complete, while the stream continues.
 // Every wait is bounded: on expiry the kernel records MKV_ERR_TIMEOUT, every role drains
 // (the producer waits, bounded again, for its copies in flight) and the CTA returns.
 #include <cstdlib>
@@ -87,8 +86,7 @@ struct Control {
     StageMeta meta[kMaxStages];
     ExchangeRef xq[kMaxStages];
     int abort_flag;
-    int tail_entry;    // queue index the tail warps hold, or -1
-    int tail_unit;
+    int tail_unit;     // unit whose tail is due, or -1
 };
 
 constexpr size_t smem_bytes(int nst) {
@@ -139,7 +137,6 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             ptx::mbar_init(ptx::smem_u32(&ctl->qempty[s]), kConsumerWarps);
         }
         ctl->abort_flag = 0;
-        ctl->tail_entry = -1;
         ctl->tail_unit = -1;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async();
@@ -528,58 +525,41 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             if (lane < kConsumerWarps) ptx::mbar_arrive(ptx::smem_u32(&ctl->empty[ref.stage]));
             __threadfence();
             __syncwarp();
-            if (lane == 0) {
-                MKV_TR(4);
-                // the delivery that completes the unit's tile count makes its tail due
-                if (atomicAdd(&L.done[u], ref.ntiles) + ref.ntiles == ref.total) {
-                    const int idx = atomicAdd(&L.tq_pub[0], 1);
-                    if (idx < L.n_units) {
-                        L.tq_unit[idx] = u;
-                        __threadfence();
-                        atomicExch(&L.tq_ready[idx], 1);
-                    } else {
-                        atomicCAS(p.status, kStatusOk, kStatusDeviceCheck);
-                    }
-                }
-            }
+            // The tail group that looks after this unit watches the count; nothing to announce.
+            if (lane == 0) { MKV_TR(4); atomicAdd(&L.done[u], ref.ntiles); }
         }
     } else {
         // ================================ tail warps ===================================
-        // Unit tails are served from one queue per layer: each tail group claims the next
-        // queue index and waits for that entry to be published, so every due tail finds an
-        // idle group of its own and no CTA ever has two to run.  Groups whose index lies
-        // beyond the number of units have nothing to wait for.
+        // Unit tails are spread statically: this CTA's tail group looks after units
+        // blockIdx.x, blockIdx.x + gridDim.x, ...  It watches the unit's count of delivered
+        // tiles and runs the tail the moment the count is complete, so no CTA ever has two
+        // tails due at once (as long as there are at least as many CTAs as units) and nothing
+        // has to be announced or claimed.
         ptx::griddep_wait();
         const int tt = tid - kTailTid0;
-        for (;;) {
+        for (int u = blockIdx.x; u < L.n_units; u += gridDim.x) {
             if (tt == 0) {
-                int my = atomicAdd(&L.tq_claim[0], 1), unit = -1;
-                if (my < L.n_units) {
-                    const unsigned long long t0 = ptx::globaltimer_ns();
-                    for (;;) {
-                        if (*reinterpret_cast<volatile int*>(&L.tq_ready[my]) != 0) { __threadfence(); unit = __ldcg(&L.tq_unit[my]); break; }
-                        if (aborted(ctl)) break;
-                        if (ptx::globaltimer_ns() - t0 > kWaitNs) { note_timeout(p, ctl); break; }
-                        __nanosleep(200);
-                    }
+                const int total = unit_tiles(L.unit_lp[u], min(L.n_dec[u], p.cap - (dec ? 1 : 0)));
+                const unsigned long long t0 = ptx::globaltimer_ns();
+                int okk = 0;
+                for (;;) {
+                    if (*reinterpret_cast<volatile int*>(&L.done[u]) >= total) { okk = 1; break; }
+                    if (aborted(ctl)) break;
+                    if (ptx::globaltimer_ns() - t0 > kWaitNs) { note_timeout(p, ctl); break; }
+                    __nanosleep(100);
                 }
-                ctl->tail_entry = unit >= 0 ? my : -1;
-                ctl->tail_unit = unit;
+                ctl->tail_unit = okk ? u : -1;
             }
             bar_sync(1, kTailThreads);
-            const int my = ctl->tail_entry, u = ctl->tail_unit;
-            bar_sync(1, kTailThreads);     // everyone has read them before thread 0 writes again
-            if (my < 0) break;
+            const int got = ctl->tail_unit;
+            bar_sync(1, kTailThreads);     // everyone has read it before thread 0 writes again
+            if (got < 0) break;
+            __threadfence();
             if (tt == 0) MKV_TR_ADD(6, 1);
             const TailJob job = load_tail_job(L, u);
             if (G <= 4) unit_tail<__nv_bfloat16, kTailThreads, 1, 4>(p, job, *tsm, tt);
             else unit_tail<__nv_bfloat16, kTailThreads, 1, 8>(p, job, *tsm, tt);
-            // rewind the idle copy of the queue for the launch after next
-            if (tt == 0) {
-                L.tq_ready_idle[my] = 0;
-                if (my == 0) { L.tq_claim_idle[0] = 0; L.tq_pub_idle[0] = 0; }
-                MKV_TR(5);
-            }
+            if (tt == 0) MKV_TR(5);
         }
     }
 }
