@@ -23,7 +23,7 @@ inline int elem_size(int dt) { return dt == MKV_BF16 ? 2 : 4; }
 
 struct LayerOff {
     size_t Kp, Vp, Kd, Vd, score, pos, n_dec, abar, n_prev, ev_k, ev_pos, ev_score, cta_unit0, cta_head0,
-        cta_headn, unit_lp, unit_next0, next, done, nslots, unit_step, end;
+        cta_headn, unit_lp, unit_next0, next, cnt, unit_step, end;
 };
 // Scratch that lives for one step only, shared by all layers of the context (calls on a
 // context are ordered on one stream, and a step touches it only after every earlier kernel
@@ -88,8 +88,7 @@ bool make_layout(int layers, int batch, int q_heads, int kv_heads, int head_dim,
     L.lo.unit_lp = take(U * 4);
     L.lo.unit_next0 = take(U * 4);
     L.lo.next = take(2 * U * 4);      // two copies each, alternating from launch to launch
-    L.lo.done = take(2 * U * 4);
-    L.lo.nslots = take(2 * U * 4);
+    L.lo.cnt = take(2 * U * 8);
     L.lo.unit_step = take(U * 4);
     L.lo.end = o;
     L.layer_bytes = o;
@@ -169,11 +168,9 @@ LayerDev layer_dev(const mkv_ctx* c, int layer) {
     d.unit_lp = (const int32_t*)(base + o.unit_lp);
     d.unit_next0 = (const int32_t*)(base + o.unit_next0);
     d.next = (int32_t*)(base + o.next) + cur * U;
-    d.done = (int32_t*)(base + o.done) + cur * U;
-    d.nslots = (int32_t*)(base + o.nslots) + cur * U;
+    d.cnt = (int2*)(base + o.cnt) + cur * U;
     d.next_idle = (int32_t*)(base + o.next) + idle * U;
-    d.done_idle = (int32_t*)(base + o.done) + idle * U;
-    d.nslots_idle = (int32_t*)(base + o.nslots) + idle * U;
+    d.cnt_idle = (int2*)(base + o.cnt) + idle * U;
     d.part_o = (float*)(sb + so.part_o);
     d.part_ml = (float*)(sb + so.part_ml);
     d.unit_step = (int32_t*)(base + o.unit_step);
@@ -358,8 +355,7 @@ mkv_status mkv_prefill(mkv_ctx* c, int layer, const void* K, const void* V, cons
     ok &= cudaMemcpyAsync(base + L.lo.unit_next0, next0.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok &= cudaMemcpyAsync(base + L.lo.next, next0.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok &= cudaMemcpyAsync(base + L.lo.next + (size_t)U * 4, next0.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok &= cudaMemsetAsync(base + L.lo.done, 0, 2 * (size_t)U * 4, st) == cudaSuccess;
-    ok &= cudaMemsetAsync(base + L.lo.nslots, 0, 2 * (size_t)U * 4, st) == cudaSuccess;
+    ok &= cudaMemsetAsync(base + L.lo.cnt, 0, 2 * (size_t)U * 8, st) == cudaSuccess;
     // empty decode pool, rewind counters
     ok &= cudaMemsetAsync(base + L.lo.n_dec, 0, U * 4, st) == cudaSuccess;
     ok &= cudaMemsetAsync(base + L.lo.n_prev, 0, U * 4, st) == cudaSuccess;

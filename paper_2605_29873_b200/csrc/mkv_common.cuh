@@ -72,11 +72,9 @@ struct LayerDev {
     const int32_t* unit_lp;     // [units] prefill length
     const int32_t* unit_next0;  // [units] tiles reserved in the unit = start value of its counter
     int32_t* next;     // [units] tiles handed out so far (this launch's copy)
-    int32_t* done;     // [units] tiles delivered so far
-    int32_t* nslots;   // [units] partial slots taken so far
+    int2* cnt;         // [units] x: tiles delivered so far, y: partial slots taken so far
     int32_t* next_idle;   // the other copies, rewound by the tails for the next launch
-    int32_t* done_idle;
-    int32_t* nslots_idle;
+    int2* cnt_idle;
     float* part_o;     // [units][kMaxParts][G][d]
     float* part_ml;    // [units][kMaxParts][G][2]  (running max in log2 units, running sum)
     int32_t* unit_step;// [units] decode steps completed

@@ -86,7 +86,7 @@ struct Control {
     StageMeta meta[kMaxStages];
     ExchangeRef xq[kMaxStages];
     int abort_flag;
-    int tail_unit;     // unit whose tail is due, or -1
+    int tail_unit;     // partial slots of the unit whose tail is due, or -1
 };
 
 constexpr size_t smem_bytes(int nst) {
@@ -110,6 +110,41 @@ __device__ inline bool wait_or_abort(uint32_t bar, uint32_t parity, Control* ctl
             if (ptx::mbar_try_wait(bar, parity)) return true;
         if (aborted(ctl)) return false;
         if (ptx::globaltimer_ns() - t0 > kWaitNs) return false;
+    }
+}
+
+// The tail warps' loop over the units this CTA looks after.  While a unit is still being
+// streamed the group already fetches what its tail needs and the step does not change
+// (tail_prefetch); thread 0 then watches the unit's counters, which arrive as one 8-byte
+// word (tiles delivered, partial slots taken).
+template <int GB>
+__device__ void tail_group(const Params& p, Control* ctl, TailSmem<kTailThreads>* tsm, int tt) {
+    const LayerDev& L = p.L;
+    const bool dec = (p.mode == kModeDecode);
+    for (int u = blockIdx.x; u < L.n_units; u += gridDim.x) {
+        TailPre<kTailThreads, GB> pre;
+        tail_prefetch<__nv_bfloat16, kTailThreads, GB>(p, u, *tsm, tt, pre);
+        if (tt == 0) {
+            const int total = unit_tiles(L.unit_lp[u], min(pre.n_dec, p.cap - (dec ? 1 : 0)));
+            const unsigned long long t0 = ptx::globaltimer_ns();
+            int slots = -1;
+            for (;;) {
+                const unsigned long long w = *reinterpret_cast<const volatile unsigned long long*>(&L.cnt[u]);
+                if ((int)(unsigned)(w & 0xffffffffull) >= total) { slots = (int)(unsigned)(w >> 32); break; }
+                if (aborted(ctl)) break;
+                if (ptx::globaltimer_ns() - t0 > kWaitNs) { note_timeout(p, ctl); break; }
+                __nanosleep(100);
+            }
+            ctl->tail_unit = slots;
+        }
+        bar_sync(1, kTailThreads);
+        const int slots = ctl->tail_unit;
+        bar_sync(1, kTailThreads);     // everyone has read it before thread 0 writes again
+        if (slots < 0) break;
+        __threadfence();
+        if (tt == 0) MKV_TR_ADD(6, 1);
+        unit_tail<__nv_bfloat16, kTailThreads, 1, GB>(p, u, slots, pre, *tsm, tt);
+        if (tt == 0) MKV_TR(5);
     }
 }
 
@@ -234,7 +269,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         int total = unit_tiles(lp, n_old);
         int chunk = unit_chunk(total);
         if (lane == 0 && ok && head_end > L.cta_head0[blockIdx.x]) {
-            slot = atomicAdd(&L.nslots[u], 1);
+            slot = atomicAdd(&L.cnt[u].y, 1);
             ok = issue_query(u);
             q_sent = true;
             for (; head_t < head_end && ok; ++head_t) {
@@ -251,7 +286,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             if (g < total) {
                 if (lane == 0) {
                     const int g_next = atomicAdd(&L.next[u], chunk);   // in flight while this chunk is issued
-                    if (slot < 0) slot = atomicAdd(&L.nslots[u], 1);
+                    if (slot < 0) slot = atomicAdd(&L.cnt[u].y, 1);
                     const int t_end = min(g + chunk, total);
                     for (int t = g; t < t_end && ok; ++t) {
                         const TileRef tr = tile_ref(t, lp, n_old);
@@ -526,7 +561,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             __threadfence();
             __syncwarp();
             // The tail group that looks after this unit watches the count; nothing to announce.
-            if (lane == 0) { MKV_TR(4); atomicAdd(&L.done[u], ref.ntiles); }
+            if (lane == 0) { MKV_TR(4); atomicAdd(&L.cnt[u].x, ref.ntiles); }
         }
     } else {
         // ================================ tail warps ===================================
@@ -536,31 +571,8 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         // tails due at once (as long as there are at least as many CTAs as units) and nothing
         // has to be announced or claimed.
         ptx::griddep_wait();
-        const int tt = tid - kTailTid0;
-        for (int u = blockIdx.x; u < L.n_units; u += gridDim.x) {
-            if (tt == 0) {
-                const int total = unit_tiles(L.unit_lp[u], min(L.n_dec[u], p.cap - (dec ? 1 : 0)));
-                const unsigned long long t0 = ptx::globaltimer_ns();
-                int okk = 0;
-                for (;;) {
-                    if (*reinterpret_cast<volatile int*>(&L.done[u]) >= total) { okk = 1; break; }
-                    if (aborted(ctl)) break;
-                    if (ptx::globaltimer_ns() - t0 > kWaitNs) { note_timeout(p, ctl); break; }
-                    __nanosleep(100);
-                }
-                ctl->tail_unit = okk ? u : -1;
-            }
-            bar_sync(1, kTailThreads);
-            const int got = ctl->tail_unit;
-            bar_sync(1, kTailThreads);     // everyone has read it before thread 0 writes again
-            if (got < 0) break;
-            __threadfence();
-            if (tt == 0) MKV_TR_ADD(6, 1);
-            const TailJob job = load_tail_job(L, u);
-            if (G <= 4) unit_tail<__nv_bfloat16, kTailThreads, 1, 4>(p, job, *tsm, tt);
-            else unit_tail<__nv_bfloat16, kTailThreads, 1, 8>(p, job, *tsm, tt);
-            if (tt == 0) MKV_TR(5);
-        }
+        if (G <= 4) tail_group<4>(p, ctl, tsm, tid - kTailTid0);
+        else tail_group<8>(p, ctl, tsm, tid - kTailTid0);
     }
 }
 

@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
         }
         if (mine > 0) {
             // merge the four warps, write the visit's partial into a fresh slot of the unit
-            if (tid == 0) s_g = atomicAdd(&L.nslots[u], 1);
+            if (tid == 0) s_g = atomicAdd(&L.cnt[u].y, 1);
             if (lane == 0) {
 #pragma unroll
                 for (int h = 0; h < G; ++h) { xm[warp][h] = m[h]; xl[warp][h] = l[h]; }
@@ -168,11 +168,14 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
             __threadfence();
             __syncthreads();
             // the delivery that completes the unit's tile count runs its tail
-            if (tid == 0) s_last = (atomicAdd(&L.done[u], mine) + mine == total);
+            if (tid == 0) s_last = (atomicAdd(&L.cnt[u].x, mine) + mine == total);
             __syncthreads();
             if (s_last) {
                 __threadfence();
-                unit_tail<T, kSimtThreads, 1, (G <= 4 ? 4 : 8)>(p, load_tail_job(L, u), tsm, tid);
+                constexpr int GB = G <= 4 ? 4 : 8;
+                TailPre<kSimtThreads, GB> pre;
+                tail_prefetch<T, kSimtThreads, GB>(p, u, tsm, tid, pre);
+                unit_tail<T, kSimtThreads, 1, GB>(p, u, __ldcg(&L.cnt[u].y), pre, tsm, tid);
             }
             __syncthreads();
         }

@@ -81,22 +81,25 @@ __device__ inline void load_elems(const T* ptr, float (&f)[N]) {
     }
 }
 
-// What a tail needs to know about its unit.  Whoever takes the last ticket loads it (the
-// loads overlap that thread's other work) and hands it over.
-struct TailJob { int u, P, part0, n_dec, t; };
-
-__device__ inline TailJob load_tail_job(const LayerDev& L, int u) {
-    TailJob j;
-    j.u = u; j.P = min(__ldcg(&L.nslots[u]), kMaxParts); j.part0 = u * kMaxParts; j.n_dec = L.n_dec[u]; j.t = L.unit_step[u];
-    return j;
-}
-
 // The unit is complete: prepare the idle copy of its counters for the next launch.
 __device__ inline void rewind_unit(const LayerDev& L, int u) {
     L.next_idle[u] = L.unit_next0[u];
-    L.done_idle[u] = 0;
-    L.nslots_idle[u] = 0;
+    L.cnt_idle[u] = make_int2(0, 0);
 }
+
+// What a tail can fetch before its unit is complete (nothing here is written by the step
+// until the tail itself runs): the unit's decode count and step number, the scores and
+// position ids of the tokens this thread will handle in the first two passes, and the fresh
+// token's value elements; the fresh token's logits go to shared memory.
+template <int NT, int GB>
+struct TailPre {
+    static constexpr int TW = GB <= 4 ? 4 : 2;          // tokens per thread and pass (one 16- or 8-byte vector)
+    static constexpr int OCB = (GB * 32 + NT - 1) / NT; // float4 output elements per thread (bound)
+    int n_dec, t;
+    float sc[2][TW];
+    int ps[2][TW];
+    float vn[OCB][4];
+};
 
 __device__ inline void store_out4(const Params& p, size_t idx, float4 v) {
     if (p.out_f32) {
@@ -110,27 +113,91 @@ __device__ inline void store_out4(const Params& p, size_t idx, float4 v) {
     }
 }
 
+template <int TW>
+__device__ inline void load_vec(const float* src, float (&dst)[TW]) {
+    if constexpr (TW == 4) {
+        const float4 v = __ldcg(reinterpret_cast<const float4*>(src));
+        dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+    } else {
+        const float2 v = __ldcg(reinterpret_cast<const float2*>(src));
+        dst[0] = v.x; dst[1] = v.y;
+    }
+}
+template <int TW>
+__device__ inline void load_vec(const int32_t* src, int (&dst)[TW]) {
+    float f[TW];
+    load_vec<TW>(reinterpret_cast<const float*>(src), f);
+#pragma unroll
+    for (int j = 0; j < TW; ++j) dst[j] = __float_as_int(f[j]);
+}
+
 // GB: compile-time bound of the group size G (4 or 8); it sizes the register staging.
-template <typename T, int NT, int BAR, int GB>
-__device__ void unit_tail(const Params& p, const TailJob& job, TailSmem<NT>& sm, int tid) {
+template <typename T, int NT, int GB>
+__device__ void tail_prefetch(const Params& p, int u, TailSmem<NT>& sm, int tid, TailPre<NT, GB>& pre) {
+    constexpr int TW = TailPre<NT, GB>::TW, OCB = TailPre<NT, GB>::OCB, NW = NT / 32;
     const LayerDev& L = p.L;
-    const int u = job.u;
+    const int G = p.group, D = p.head_dim, ls = p.lstride;
+    const int b = u / p.kv_heads, g = u - b * p.kv_heads;
+    const int lane = tid & 31, warp = tid >> 5;
+    const bool dec = (p.mode == kModeDecode);
+    pre.n_dec = L.n_dec[u];
+    pre.t = L.unit_step[u];
+    if (!dec) return;
+    const T* qrow = reinterpret_cast<const T*>(p.q) + ((size_t)b * p.q_heads + (size_t)g * G) * D;
+    const T* knew = reinterpret_cast<const T*>(p.k_new) + (size_t)u * D;
+    const T* vnew = reinterpret_cast<const T*>(p.v_new) + (size_t)u * D;
+    const float* score = L.score + (size_t)u * ls;
+    const int32_t* pos = L.pos + (size_t)u * ls;
+    const int n_old = min(pre.n_dec, p.cap - 1);
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        const int i0 = TW * (tid + k * NT);
+        if (i0 < n_old) { load_vec<TW>(score + i0, pre.sc[k]); load_vec<TW>(pos + i0, pre.ps[k]); }
+    }
+    const int ne = G * D / 4;
+#pragma unroll
+    for (int c = 0; c < OCB; ++c) {
+        const int e = tid + c * NT;
+        if (e < ne) load_elems<T, 4>(vnew + (4 * e) % D, pre.vn[c]);
+    }
+    // logit of the fresh token: lane l holds D/32 consecutive elements
+    for (int h = warp; h < G; h += NW) {
+        float a = 0.f;
+        if (D == 128) {
+            float qv[4], kv[4];
+            load_elems<T, 4>(qrow + (size_t)h * D + 4 * lane, qv);
+            load_elems<T, 4>(knew + 4 * lane, kv);
+            a = fmaf(qv[0], kv[0], fmaf(qv[1], kv[1], fmaf(qv[2], kv[2], qv[3] * kv[3])));
+        } else {
+            float qv[2], kv[2];
+            load_elems<T, 2>(qrow + (size_t)h * D + 2 * lane, qv);
+            load_elems<T, 2>(knew + 2 * lane, kv);
+            a = fmaf(qv[0], kv[0], qv[1] * kv[1]);
+        }
+#pragma unroll
+        for (int off = 16; off; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
+        if (lane == 0) sm.snew[h] = a * p.scale_log2;
+    }
+}
+
+// The tail proper; P = partial slots the unit's visits took.
+template <typename T, int NT, int BAR, int GB>
+__device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB>& pre, TailSmem<NT>& sm, int tid) {
+    const LayerDev& L = p.L;
     const int G = p.group, D = p.head_dim, cap = p.cap, ls = p.lstride;
     const int rowb = D * (int)sizeof(T);
     const int b = u / p.kv_heads, g = u - b * p.kv_heads;
-    const int P = job.P, part0 = job.part0;
+    const int P = min(P_in, kMaxParts), part0 = u * kMaxParts;
     const bool dec = (p.mode == kModeDecode);
-    const int n_old = min(job.n_dec, dec ? cap - 1 : cap);
+    const int n_old = min(pre.n_dec, dec ? cap - 1 : cap);
     const int n = dec ? n_old + 1 : n_old;
-    const int t = job.t;
+    const int t = pre.t;
     const int lane = tid & 31, warp = tid >> 5;
     constexpr int NW = NT / 32;
-    constexpr int TW = GB <= 4 ? 4 : 2;                 // tokens per thread and pass (one 16- or 8-byte vector)
-    constexpr int TV = 1;                               // token vectors per thread loaded up front
+    constexpr int TW = TailPre<NT, GB>::TW;
     constexpr int PB = GB <= 4 ? 2 : 1;                 // partials staged in registers up front
     constexpr int LB = 4;                               // partials fetched per trip after those
-    constexpr int OCB = (GB * 32 + NT - 1) / NT;        // float4 output elements per thread (bound)
-    const T* qrow = reinterpret_cast<const T*>(p.q) + ((size_t)b * p.q_heads + (size_t)g * G) * D;
+    constexpr int OCB = TailPre<NT, GB>::OCB;
     const T* knew = reinterpret_cast<const T*>(p.k_new) + (size_t)u * D;
     const T* vnew = reinterpret_cast<const T*>(p.v_new) + (size_t)u * D;
     float* score = L.score + (size_t)u * ls;
@@ -142,36 +209,19 @@ __device__ void unit_tail(const Params& p, const TailJob& job, TailSmem<NT>& sm,
     if (tid == 0) MKV_TR(8);
 
     // Everything below is latency: a few dependent trips to L2.  So every load that does
-    // not need the softmax statistics is issued first, in one batch: this thread's tokens'
-    // logits, scores and position ids (one vector each), its share of the first partials'
-    // O, the fresh token's value and dot products, and the partials' (m, l).
-    struct Tok { float lgv[GB][TW]; float sc[TW]; int ps[TW]; };
-    auto load_vec = [&](const float* src, float (&dst)[TW]) {
-        if constexpr (TW == 4) {
-            const float4 v = __ldcg(reinterpret_cast<const float4*>(src));
-            dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
-        } else {
-            const float2 v = __ldcg(reinterpret_cast<const float2*>(src));
-            dst[0] = v.x; dst[1] = v.y;
-        }
-    };
+    // not need the softmax statistics is issued first, in one batch: the logits of this
+    // thread's tokens (first two passes), its share of the first partials' O, and the
+    // partials' (m, l).
+    struct Tok { float lgv[GB][TW]; };
     auto load_tok = [&](int i0, Tok& r) {
         if (i0 < n_old) {
 #pragma unroll
             for (int h = 0; h < GB; ++h)
-                if (h < G) load_vec(lg + (size_t)h * ls + i0, r.lgv[h]);
-            load_vec(score + i0, r.sc);
-            float pf[TW];
-            load_vec(reinterpret_cast<const float*>(pos + i0), pf);
-#pragma unroll
-            for (int j = 0; j < TW; ++j) r.ps[j] = __float_as_int(pf[j]);
+                if (h < G) load_vec<TW>(lg + (size_t)h * ls + i0, r.lgv[h]);
         }
     };
-    Tok tk[TV];
-    if (dec) {
-#pragma unroll
-        for (int v = 0; v < TV; ++v) load_tok(TW * (tid + v * NT), tk[v]);
-    }
+    Tok tk;
+    if (dec) load_tok(TW * tid, tk);
     float4 po[PB][OCB];
 #pragma unroll
     for (int q = 0; q < PB; ++q)
@@ -187,32 +237,6 @@ __device__ void unit_tail(const Params& p, const TailJob& job, TailSmem<NT>& sm,
             const float2 ml = __ldcg(reinterpret_cast<const float2*>(&L.part_ml[((size_t)(part0 + q) * G + h) * 2]));
             sm.w[q][h] = ml.x;
             sm.pl[q][h] = ml.y;
-        }
-    }
-    // ---- 0. the fresh token: its value row and its logit (lane l holds D/32 consecutive elements)
-    float vn[OCB][4];
-    if (dec) {
-#pragma unroll
-        for (int c = 0; c < OCB; ++c) {
-            const int e = tid + c * NT;
-            if (e < ne) load_elems<T, 4>(vnew + (4 * e) % D, vn[c]);
-        }
-        for (int h = warp; h < G; h += NW) {
-            float a = 0.f;
-            if (D == 128) {
-                float qv[4], kv[4];
-                load_elems<T, 4>(qrow + (size_t)h * D + 4 * lane, qv);
-                load_elems<T, 4>(knew + 4 * lane, kv);
-                a = fmaf(qv[0], kv[0], fmaf(qv[1], kv[1], fmaf(qv[2], kv[2], qv[3] * kv[3])));
-            } else {
-                float qv[2], kv[2];
-                load_elems<T, 2>(qrow + (size_t)h * D + 2 * lane, qv);
-                load_elems<T, 2>(knew + 2 * lane, kv);
-                a = fmaf(qv[0], kv[0], qv[1] * kv[1]);
-            }
-#pragma unroll
-            for (int off = 16; off; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
-            if (lane == 0) sm.snew[h] = a * p.scale_log2;
         }
     }
     if (tid == 0) MKV_TR(9);
@@ -246,7 +270,7 @@ __device__ void unit_tail(const Params& p, const TailJob& job, TailSmem<NT>& sm,
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         if (dec) {
             const float wn = sm.wnew[h];
-            acc = make_float4(vn[c][0] * wn, vn[c][1] * wn, vn[c][2] * wn, vn[c][3] * wn);
+            acc = make_float4(pre.vn[c][0] * wn, pre.vn[c][1] * wn, pre.vn[c][2] * wn, pre.vn[c][3] * wn);
         }
 #pragma unroll
         for (int q = 0; q < PB; ++q) {
@@ -301,7 +325,7 @@ __device__ void unit_tail(const Params& p, const TailJob& job, TailSmem<NT>& sm,
     const unsigned long long key_new = ((unsigned long long)__float_as_uint(ab_new) << 32) | (unsigned)t;
     unsigned long long best_key = ~0ull;
     int best_slot = -1;
-    auto process_tok = [&](int i0, const Tok& r) {
+    auto process_tok = [&](int i0, const Tok& r, const float (&sc)[TW], const int (&ps)[TW]) {
         if (i0 >= n_old) return;
         float ab[TW], nw[TW];
 #pragma unroll
@@ -317,7 +341,7 @@ __device__ void unit_tail(const Params& p, const TailJob& job, TailSmem<NT>& sm,
 #pragma unroll
         for (int j = 0; j < TW; ++j) {
             ab[j] *= inv_g;
-            nw[j] = fmaf(p.beta, r.sc[j], ab[j]);
+            nw[j] = fmaf(p.beta, sc[j], ab[j]);
         }
         if (i0 + TW <= n_old) {
             if constexpr (TW == 4) *reinterpret_cast<float4*>(score + i0) = make_float4(nw[0], nw[1], nw[2], nw[3]);
@@ -330,21 +354,29 @@ __device__ void unit_tail(const Params& p, const TailJob& job, TailSmem<NT>& sm,
         for (int j = 0; j < TW; ++j) {
             if (i0 + j < n_old) {
                 if (L.abar) L.abar[(size_t)u * cap + i0 + j] = ab[j];
-                const unsigned long long key = ((unsigned long long)__float_as_uint(nw[j]) << 32) | (unsigned)r.ps[j];
+                const unsigned long long key = ((unsigned long long)__float_as_uint(nw[j]) << 32) | (unsigned)ps[j];
                 if (k > 1) keys[i0 + j] = key;
                 if (key < best_key) { best_key = key; best_slot = i0 + j; }
             }
         }
     };
-#pragma unroll
-    for (int v = 0; v < TV; ++v) process_tok(TW * (tid + v * NT), tk[v]);
+    process_tok(TW * tid, tk, pre.sc[0], pre.ps[0]);
     // further passes; the rest of `out` travels with the first of them (one trip, not two)
     bool out_done = false;
-    for (int base = TV * TW * NT; base < n_old; base += TW * NT) {
+    for (int base = TW * NT, pass = 1; base < n_old; base += TW * NT, ++pass) {
         const int i0 = base + TW * tid;
-        load_tok(i0, tk[0]);
+        load_tok(i0, tk);
+        float sc[TW];
+        int ps[TW];
+        if (pass == 1) {
+#pragma unroll
+            for (int j = 0; j < TW; ++j) { sc[j] = pre.sc[1][j]; ps[j] = pre.ps[1][j]; }
+        } else if (i0 < n_old) {
+            load_vec<TW>(score + i0, sc);
+            load_vec<TW>(pos + i0, ps);
+        }
         if (!out_done) { finish_out(); out_done = true; }
-        process_tok(i0, tk[0]);
+        process_tok(i0, tk, sc, ps);
     }
     if (!out_done) finish_out();
     if (tid == 0) MKV_TR(12);
