@@ -56,3 +56,154 @@ def test_llama_layer_bf16_reduced(kernel):
     assert rep.ok(), rep.failures[:5]
     assert rep.max_out_err <= 2e-3 and rep.max_score_err <= 1e-4
     assert rep.evicted_not_newest > 20
+
+
+def test_ragged_batch_bf16():
+    """Headline shape reduced: several sequences with different prefill lengths (ragged tails in
+    both pools, units of different size sharing the CTAs), tensor-core kernel."""
+    w = CONFIGS["llama_b16"].with_(batch=5, prefill=(90, 700), steps=300, budget=140, variant="hot", n_heavy=4)
+    rep = run_case(w, w.steps, check_every=3)
+    assert rep.ok(), rep.failures[:5]
+    assert rep.max_out_err <= 2e-3 and rep.max_score_err <= 1e-4
+    assert rep.evicted_not_newest > 50
+
+
+def test_qwen_group7_bf16():
+    """GQA group 7 (28 query heads on 4 KV heads): the padded head rows of the tensor-core
+    kernel and the 8-head staging of the tail."""
+    w = CONFIGS["qwen_b64"].with_(batch=3, prefill=210, steps=240, budget=100, variant="hot", n_heavy=4)
+    rep = run_case(w, w.steps, check_every=2)
+    assert rep.ok(), rep.failures[:5]
+    assert rep.max_out_err <= 2e-3 and rep.max_score_err <= 1e-4
+    assert rep.evicted_not_newest > 20
+
+
+def test_empty_prefill_and_bf16_out_through_host_api():
+    """No prompt at all (the decode pool is the whole cache), bf16 output, host-buffer entry
+    point: covers the unit with nothing cached at the first step."""
+    w = CONFIGS["llama_b1"].with_(prefill=0, steps=150, budget=40, variant="hot", n_heavy=2)
+    ctx = make_context(w, out_f32=False)
+    stream = BatchStream(w, 0)
+    oracles, _ = prefill_both(ctx, w, stream)
+    rep = lockstep(ctx, w, stream, oracles, w.steps, host_api=True)
+    ctx.close()
+    assert rep.ok(), rep.failures[:5]
+    assert rep.evictions == (w.steps - w.budget) * w.kv_heads
+
+
+@pytest.mark.parametrize("kernel", [mkv.MKV_KERNEL_SIMT, mkv.MKV_KERNEL_AUTO])
+def test_budget_shrink_evicts_many_at_once(kernel):
+    """mkv_set_budget below the current count: the next step evicts overflow > 1 tokens (the
+    general arg-min of Eq. 8: radix select, ordered hole filling)."""
+    w = CONFIGS["llama_b1"].with_(prefill=130, steps=200, budget=120, variant="hot", n_heavy=3)
+    ctx = make_context(w, kernel=kernel)
+    stream = BatchStream(w, 0)
+    oracles, _ = prefill_both(ctx, w, stream)
+    rep = lockstep(ctx, w, stream, oracles, 150)
+    ctx.set_budget(67)
+    for o in oracles:
+        o.set_budget(67)
+    rep = lockstep(ctx, w, stream, oracles, 50, report=rep)
+    for g in range(w.kv_heads):
+        pos, _ = ctx.decode_state(0, 0, g)
+        assert len(pos) == 67
+    ctx.close()
+    assert rep.ok(), rep.failures[:5]
+    assert rep.max_out_err <= 2e-3 and rep.max_score_err <= 1e-4
+
+
+def test_two_layers_keep_independent_state():
+    """Steps on two layers interleaved (each layer has its own pools, scores and counters)."""
+    w = CONFIGS["llama_b1"].with_(prefill=200, steps=120, budget=50, variant="hot", n_heavy=2)
+    ctx = make_context(w, layers=2)
+    streams = [BatchStream(w.with_(seed=s), 0) for s in (0, 1)]
+    oracles = [prefill_both(ctx, w, streams[l], layer=l)[0] for l in (0, 1)]
+    reps = [ParityReport(), ParityReport()]
+    for _ in range(6):
+        for l in (0, 1):
+            lockstep(ctx, w, streams[l], oracles[l], 20, layer=l, report=reps[l], chunk=20)
+    ctx.close()
+    for rep in reps:
+        assert rep.ok(), rep.failures[:5]
+        assert rep.steps == 120 and rep.evictions > 0
+
+
+def attention_f64(q, K, V, G):
+    """softmax(q K^T / sqrt(d)) V written out in numpy fp64; q [Hq,d], K/V [Hkv,N,d]."""
+    d = q.shape[-1]
+    out = np.zeros_like(q)
+    probs = []
+    for h in range(q.shape[0]):
+        s = K[h // G] @ q[h] / np.sqrt(d)
+        e = np.exp(s - s.max())
+        pr = e / e.sum()
+        probs.append(pr)
+        out[h] = pr @ V[h // G]
+    return out, probs
+
+
+def test_headline_shape_sampled_units_at_steady_state():
+    """The bench's own configuration (llama_b16: batch 16, prefill U[512,4096], budget 1024, the
+    grid and chunking the bench times), run to steady state with device-generated inputs.  One
+    further step is then checked on sampled (sequence, KV head) units against the definitions
+    computed from the GPU's own pre-step state: attention over prefill + pool + fresh token,
+    Eq. 4-5 scores, and the oracle's select() for the evicted token."""
+    import torch
+    from oracle import mkv_oracle as O
+    w = CONFIGS["llama_b16"]
+    lens = w.prefill_lens()
+    B, Hq, Hkv, d, G = w.batch, w.q_heads, w.kv_heads, w.head_dim, w.group
+    dev = torch.device("cuda", 0)
+    ctx = mkv.MomentKV(1, Hq, Hkv, d, w.budget, w.beta, B, int(lens.max()), out_dtype=mkv.MKV_F32)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(11)
+    K = (torch.randn((B, Hkv, int(lens.max()), d), generator=gen, device=dev) / d ** 0.5).bfloat16()
+    V = (torch.randn((B, Hkv, int(lens.max()), d), generator=gen, device=dev) / d ** 0.5).bfloat16()
+    ctx.prefill(0, K, V, lens)
+    out = torch.zeros((B, Hq, d), dtype=torch.float32, device=dev)
+    ring = 32
+    qs = (2.0 * torch.randn((ring, B, Hq, d), generator=gen, device=dev)).bfloat16()
+    ks = (torch.randn((ring, B, Hkv, d), generator=gen, device=dev) / d ** 0.5).bfloat16()
+    vs = (torch.randn((ring, B, Hkv, d), generator=gen, device=dev) / d ** 0.5).bfloat16()
+    steps = w.budget + 40
+    for i in range(steps):
+        ctx.decode_step(0, qs[i % ring], ks[i % ring], vs[i % ring], out)
+    ctx.status_sync()
+    units = [(0, 0), (3, 5), (7, 2), (15, 7), (int(np.argmax(lens)), 1), (int(np.argmin(lens)), 6)]
+    before = {}
+    for b, g in units:
+        Kp, Vp = ctx.read_kv(0, b, g, 0)
+        Kd, Vd = ctx.read_kv(0, b, g, 1)
+        pos, sc = ctx.decode_state(0, b, g)
+        assert len(pos) == w.budget
+        before[(b, g)] = (Kp, Vp, Kd, Vd, pos, sc)
+    i = steps
+    ctx.decode_step(0, qs[i % ring], ks[i % ring], vs[i % ring], out)
+    ctx.status_sync()
+    got = out.double().cpu().numpy()
+    qh = qs[i % ring].double().cpu().numpy()
+    kh = ks[i % ring].double().cpu().numpy()
+    vh = vs[i % ring].double().cpu().numpy()
+    for b, g in units:
+        Kp, Vp, Kd, Vd, pos, sc = before[(b, g)]
+        Kall = np.concatenate([Kp, Kd, kh[b, g][None]])[None]
+        Vall = np.concatenate([Vp, Vd, vh[b, g][None]])[None]
+        ref, probs = attention_f64(qh[b, g * G:(g + 1) * G], Kall, Vall, G)
+        o = got[b, g * G:(g + 1) * G]
+        rowmax = np.abs(ref).max(axis=1, keepdims=True)
+        assert (np.abs(o - ref) <= 2e-3 * rowmax).all(), (b, g, np.abs(o - ref).max())
+        abar = np.mean([pr[len(Kp):] for pr in probs], axis=0)                 # Eq. 4, decode slice
+        new_sc = O.update(np.concatenate([sc.astype(np.float64), [0.0]]), abar, w.beta)   # Eq. 5, fresh token from 0
+        all_pos = np.concatenate([pos.astype(np.int64), [steps]])
+        pos2, sc2 = ctx.decode_state(0, b, g)
+        ev_pos, ev_sc = ctx.last_evicted(0, b, g)
+        assert len(pos2) == w.budget and len(ev_pos) == 1
+        g_pos = np.concatenate([pos2, ev_pos]).astype(np.int64)
+        g_sc = np.concatenate([sc2, ev_sc]).astype(np.float64)
+        assert sorted(g_pos.tolist()) == sorted(all_pos.tolist())
+        order, rorder = np.argsort(g_pos), np.argsort(all_pos)
+        rel = np.abs(g_sc[order] - new_sc[rorder]) / np.maximum(new_sc[rorder], 1e-300)
+        assert rel.max() <= 1e-4, (b, g, rel.max())
+        want = g_pos[O.select(g_sc, g_pos, 1)]            # integer selection on the GPU's own scores
+        assert want.tolist() == ev_pos.tolist()
+    ctx.close()
