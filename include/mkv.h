@@ -26,7 +26,9 @@
  *   - Errors found on the host are returned at once; errors found by a kernel
  *     (a count beyond capacity, a bounded wait that expired) set a sticky device
  *     status word that mkv_status_sync() reads.
- *   - One host thread at a time per context.
+ *   - One host thread at a time per context, and all calls of a context on one stream (or
+ *     ordered by the caller in some other way): the layers of a context share the per-step
+ *     scratch, and a step may begin while the previous kernel of its stream is still ending.
  */
 #ifndef MKV_H_
 #define MKV_H_
