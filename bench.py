@@ -217,13 +217,38 @@ def run_reference(args, w):
 
 
 def workload_config(w, lens, args):
-    return {"workload": f"{w.name}: Llama-3.1-8B attention layer shape, {w.q_heads}/{w.kv_heads} heads, "
-                        f"head_dim {w.head_dim}, {w.dtype}, batch {w.batch}, prefill lengths U[512,4096] "
+    shape = {"llama_b16": "Llama-3.1-8B attention layer shape", "llama_b1": "Llama-3.1-8B attention layer shape",
+             "llama_stack": "Llama-3.1-8B attention layer shape", "qwen_b64": "Qwen2.5-7B-like attention layer shape",
+             "tiny": "tiny single-layer shape"}.get(w.name, w.name)
+    pre = (f"prefill lengths U[{w.prefill[0]},{w.prefill[1]}]" if not isinstance(w.prefill, int) else f"prefill {w.prefill}")
+    return {"workload": f"{w.name}: {shape}, {w.q_heads}/{w.kv_heads} heads, "
+                        f"head_dim {w.head_dim}, {w.dtype}, batch {w.batch}, {pre} "
                         f"(sum {int(np.sum(lens))}), decode budget {w.budget}, beta {w.beta}, steady state "
                         f"(decode pool full, one eviction per unit per step)",
             "layers_cycled": args.layers,
             "l2": "inputs larger than L2: each layer-step streams its own ~%d MB cache, %d layers cycled"
-                  % (int(sum(w.kv_heads * (int(lp) + w.budget + 1) * ROW_BYTES for lp in lens) / 1e6), args.layers)}
+                  % (int(sum(w.kv_heads * (int(lp) + w.budget + 1) * 2 * w.head_dim * (2 if w.dtype == "bf16" else 4) for lp in lens) / 1e6), args.layers)}
+
+
+def rank_workload(w, rank):
+    """Weak scaling: every rank holds its own batch of the same shape (units are independent,
+    so the data path needs no collective); ranks differ in their seed only."""
+    return w.with_(seed=w.seed + rank)
+
+
+def max_over_ranks(times_ms, world, device):
+    """Element-wise maximum of per-rank timings (the job is as slow as its slowest rank)."""
+    import torch
+    t = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
+def job_tokens_per_s(batch, steps, world, ms_max):
+    """Whole-job throughput: tokens all ranks decoded divided by the slowest rank's time."""
+    return world * batch * steps / (ms_max * 1e-3)
 
 
 def main():
@@ -263,7 +288,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     # every rank holds its own batch (weak scaling; units are independent, no collective)
-    wr = w.with_(seed=w.seed + rank)
+    wr = rank_workload(w, rank)
     lens = wr.prefill_lens()
     Lmax = int(lens.max())
     B, Hq, Hkv, d = w.batch, w.q_heads, w.kv_heads, w.head_dim
@@ -351,14 +376,11 @@ def main():
         e2e = {"ms": ms_e2e, "steps": n_e2e, "h2d": (qs[0].numel() + ks[0].numel() + vs[0].numel()) * es,
                "d2h": hout.numel() * hout.element_size()}
 
-    t = torch.tensor([ms, ms_att, e2e["ms"] / e2e["steps"] if e2e else 0.0], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_max, ms_att_max, ms_e2e_max = (float(x) for x in t.tolist())
+    ms_max, ms_att_max, ms_e2e_max = max_over_ranks([ms, ms_att, e2e["ms"] / e2e["steps"] if e2e else 0.0], world, dev)
 
     if rank == 0:
         ms_per_step = ms_max / args.steps
-        tokens_per_s = world * B * args.steps / (ms_max * 1e-3)
+        tokens_per_s = job_tokens_per_s(B, args.steps, world, ms_max)
         peak, peak_kind = load_peaks()
         alg = algorithmic_bytes_per_step(w, lens, w.budget + 1, 1)
         achieved = alg / (ms_per_step * 1e-3) / 1e9
