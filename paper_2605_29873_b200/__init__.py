@@ -2,5 +2,5 @@
 from .mkv import (  # noqa: F401
     MKV_BF16, MKV_F32, MKV_KERNEL_AUTO, MKV_KERNEL_MMA, MKV_KERNEL_SIMT, MKV_FLAG_RECORD_PROBS,
     MKV_SCORE_GROUP_MEAN, MKV_SCORE_LAYER_MEAN, MkvError, MomentKV, load_library, workspace_bytes,
-    kv_bytes_per_token, status_string, EXPORTED_SYMBOLS, attend_noalloc,
+    kv_bytes_per_token, status_string, EXPORTED_SYMBOLS, attend_noalloc, plan_starts,
 )

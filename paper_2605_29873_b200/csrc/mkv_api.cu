@@ -118,6 +118,43 @@ __global__ void prefill_copy_kernel(const uint8_t* __restrict__ srcK, const uint
     }
 }
 
+// Start table.  A unit's rows are a sequence of 64-row tiles (prefill tiles, then decode
+// tiles); the CTAs are spread over the units in proportion to the units' tile counts (a
+// full decode pool assumed).  Each CTA owns kHeadTiles tiles outright at its place, if the
+// unit has that many prefill tiles left to give (these can be fetched before the previous
+// step has finished); everything else is handed out by the unit's counter, which
+// therefore starts behind the reserved tiles.  Returns the number of CTAs (the grid).
+int build_start_table(int batch, int kv_heads, int budget, const int32_t* prefill_lens, int n_ctas_max,
+                      std::vector<int32_t>& lp, std::vector<int32_t>& next0, std::vector<int32_t>& cta_unit0,
+                      std::vector<int32_t>& cta_head0, std::vector<int32_t>& cta_headn) {
+    const int U = batch * kv_heads;
+    const int td = ceil_div(budget, kTileRows);
+    lp.assign(U, 0);
+    next0.assign(U, 0);
+    std::vector<long long> tile_begin(U + 1, 0);
+    for (int u = 0; u < U; ++u) {
+        lp[u] = prefill_lens[u / kv_heads];
+        tile_begin[u + 1] = tile_begin[u] + ceil_div(lp[u], kTileRows) + td;
+    }
+    const long long t_all = tile_begin[U];
+    const int n_ctas = (int)std::max<long long>(1, std::min<long long>(n_ctas_max, t_all / 2));
+    cta_unit0.assign(n_ctas, 0);
+    cta_head0.assign(n_ctas, 0);
+    cta_headn.assign(n_ctas, 0);
+    int u = 0;
+    for (int cta = 0; cta < n_ctas; ++cta) {
+        const long long t0 = t_all * cta / n_ctas;
+        while (tile_begin[u + 1] <= t0) ++u;
+        cta_unit0[cta] = u;
+        if (next0[u] + kHeadTiles <= ceil_div(lp[u], kTileRows)) {
+            cta_head0[cta] = next0[u];
+            cta_headn[cta] = kHeadTiles;
+            next0[u] += kHeadTiles;
+        }
+    }
+    return n_ctas;
+}
+
 }  // namespace
 
 struct mkv_ctx {
@@ -233,6 +270,24 @@ size_t mkv_workspace_bytes(int layers, int batch, int q_heads, int kv_heads, int
     return L.total;
 }
 
+mkv_status mkv_plan_starts(int batch, int kv_heads, int budget, const int32_t* prefill_lens, int n_ctas_max,
+                           int32_t* n_ctas, int32_t* cta_unit0, int32_t* cta_head0, int32_t* cta_headn,
+                           int32_t* unit_next0) {
+    if (batch < 1 || kv_heads < 1 || budget < 1 || !prefill_lens || n_ctas_max < 1 || n_ctas_max > kMaxCtas)
+        return MKV_ERR_INVALID_ARG;
+    if (!n_ctas || !cta_unit0 || !cta_head0 || !cta_headn || !unit_next0) return MKV_ERR_INVALID_ARG;
+    for (int b = 0; b < batch; ++b)
+        if (prefill_lens[b] < 0) return MKV_ERR_INVALID_ARG;
+    std::vector<int32_t> lp, next0, u0, h0, hn;
+    const int n = build_start_table(batch, kv_heads, budget, prefill_lens, n_ctas_max, lp, next0, u0, h0, hn);
+    *n_ctas = n;
+    std::memcpy(cta_unit0, u0.data(), sizeof(int32_t) * (size_t)n);
+    std::memcpy(cta_head0, h0.data(), sizeof(int32_t) * (size_t)n);
+    std::memcpy(cta_headn, hn.data(), sizeof(int32_t) * (size_t)n);
+    std::memcpy(unit_next0, next0.data(), sizeof(int32_t) * next0.size());
+    return MKV_OK;
+}
+
 size_t mkv_kv_bytes_per_token(int layers, int kv_heads, int head_dim, int kv_dtype) {
     if (layers < 1 || kv_heads < 1 || head_dim < 1 || (kv_dtype != MKV_BF16 && kv_dtype != MKV_F32)) return 0;
     return (size_t)layers * kv_heads * 2 * head_dim * elem_size(kv_dtype);
@@ -314,35 +369,9 @@ mkv_status mkv_prefill(mkv_ctx* c, int layer, const void* K, const void* V, cons
     const Layout& L = c->lay;
     const int U = L.units;
 
-    // Start table.  A unit's rows are a sequence of 64-row tiles (prefill tiles, then decode
-    // tiles); the CTAs are spread over the units in proportion to the units' tile counts (a
-    // full decode pool assumed).  Each CTA owns kHeadTiles tiles outright at its place, if the
-    // unit has that many prefill tiles left to give (these can be fetched before the previous
-    // step has finished); everything else is handed out by the unit's counter, which
-    // therefore starts behind the reserved tiles.
-    const int td = ceil_div(c->budget_max, kTileRows);
-    std::vector<int32_t> lp(U), next0(U, 0);
-    std::vector<long long> tile_begin(U + 1, 0);
-    for (int u = 0; u < U; ++u) {
-        lp[u] = prefill_lens[u / c->kv_heads];
-        tile_begin[u + 1] = tile_begin[u] + ceil_div(lp[u], kTileRows) + td;
-    }
-    const long long t_all = tile_begin[U];
-    const int n_ctas = (int)std::max<long long>(1, std::min<long long>(c->n_ctas_max, t_all / 2));
-    std::vector<int32_t> cta_unit0(n_ctas), cta_head0(n_ctas, 0), cta_headn(n_ctas, 0);
-    {
-        int u = 0;
-        for (int cta = 0; cta < n_ctas; ++cta) {
-            const long long t0 = t_all * cta / n_ctas;
-            while (tile_begin[u + 1] <= t0) ++u;
-            cta_unit0[cta] = u;
-            if (next0[u] + kHeadTiles <= ceil_div(lp[u], kTileRows)) {
-                cta_head0[cta] = next0[u];
-                cta_headn[cta] = kHeadTiles;
-                next0[u] += kHeadTiles;
-            }
-        }
-    }
+    std::vector<int32_t> lp, next0, cta_unit0, cta_head0, cta_headn;
+    const int n_ctas = build_start_table(c->batch, c->kv_heads, c->budget_max, prefill_lens, c->n_ctas_max, lp, next0,
+                                         cta_unit0, cta_head0, cta_headn);
     c->n_ctas[layer] = n_ctas;
     for (int b = 0; b < c->batch; ++b) c->lens[layer][b] = prefill_lens[b];
 

@@ -83,3 +83,32 @@ def test_create_validates_then_fails_loudly_without_a_gpu(lib):
             mkv.MomentKV(1, 4, 1, 64, 64, 0.9, 1, 64, kv_dtype=mkv.MKV_F32)
     assert lib.mkv_decode_step(None, 0, None, None, None, None, None) == 1
     lib.mkv_destroy(None)
+
+
+def test_start_table_invariants(lib):
+    """mkv_plan_starts: CTAs are spread over the units in tile order, reserved tiles are
+    disjoint prefill tiles, and a unit's counter starts right behind them."""
+    import numpy as np
+    from workloads.synthetic import CONFIGS
+    cases = [(CONFIGS["llama_b16"].prefill_lens(), 8, 1024, 296), (np.array([64], dtype=np.int32), 1, 64, 296),
+             (np.array([0, 5, 4096], dtype=np.int32), 4, 128, 296), (np.full(64, 512, dtype=np.int32), 4, 2048, 296),
+             (np.array([100000], dtype=np.int32), 2, 16, 7)]
+    for lens, hkv, budget, nmax in cases:
+        B = len(lens)
+        u0, h0, hn, nx = mkv.plan_starts(B, hkv, budget, lens, nmax)
+        U = B * hkv
+        tiles = np.array([-(-int(lens[u // hkv]) // 64) + -(-budget // 64) for u in range(U)])
+        assert 1 <= len(u0) <= nmax and len(u0) <= max(1, tiles.sum() // 2)
+        assert (np.diff(u0) >= 0).all() and u0.min() >= 0 and u0.max() < U
+        # proportional spread: CTA c starts in the unit that holds tile position c * T / n
+        begin = np.concatenate([[0], np.cumsum(tiles)])
+        for c in range(len(u0)):
+            t0 = tiles.sum() * c // len(u0)
+            assert begin[u0[c]] <= t0 < begin[u0[c] + 1]
+        assert set(hn.tolist()) <= {0, 3}
+        for u in range(U):
+            mine = np.where(u0 == u)[0]
+            got = sorted((int(h0[c]), int(hn[c])) for c in mine if hn[c] > 0)
+            # reserved ranges tile [0, next0) without gaps, all inside the prefill tiles
+            assert [g[0] for g in got] == list(range(0, 3 * len(got), 3))
+            assert nx[u] == 3 * len(got) <= -(-int(lens[u // hkv]) // 64)
