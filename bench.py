@@ -260,6 +260,8 @@ def main():
     ap.add_argument("--config", default="llama_b16", choices=sorted(CONFIGS))
     ap.add_argument("--layers", type=int, default=4)
     ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "mma"])
+    ap.add_argument("--score-mode", default="group", choices=["group", "layer"],
+                    help="group: mean over the query heads of a KV head (headline); layer: Eq. 4 over all heads")
     ap.add_argument("--budget", type=int, default=0, help="override the workload's decode budget (profiling small cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -296,7 +298,8 @@ def main():
     kv_dtype = mkv.MKV_BF16 if w.dtype == "bf16" else mkv.MKV_F32
     tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
     ctx = mkv.MomentKV(args.layers, Hq, Hkv, d, w.budget, w.beta, B, Lmax, kv_dtype=kv_dtype, out_dtype=kv_dtype,
-                       kernel=kernel, device=local)
+                       kernel=kernel, device=local,
+                       score_mode=mkv.MKV_SCORE_LAYER_MEAN if args.score_mode == "layer" else mkv.MKV_SCORE_GROUP_MEAN)
     gen = torch.Generator(device=dev)
     gen.manual_seed(1234 + rank)
     for layer in range(args.layers):

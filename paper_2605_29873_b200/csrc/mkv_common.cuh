@@ -97,6 +97,7 @@ struct Params {
     float scale_log2;  // log2(e) / sqrt(head_dim)
     int mode;
     int out_f32;
+    int defer_tails;   // the unit tails are left to a following kernel (layer-wide score mode)
 };
 
 // byte offset inside a stored row of logical byte `byte` for the row in slot `slot`

@@ -570,6 +570,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         // tiles and runs the tail the moment the count is complete, so no CTA ever has two
         // tails due at once (as long as there are at least as many CTAs as units) and nothing
         // has to be announced or claimed.
+        if (p.defer_tails) return;     // a following kernel scores the whole layer at once
         ptx::griddep_wait();
         if (G <= 4) tail_group<4>(p, ctl, tsm, tid - kTailTid0);
         else tail_group<8>(p, ctl, tsm, tid - kTailTid0);

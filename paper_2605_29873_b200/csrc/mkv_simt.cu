@@ -170,7 +170,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
             // the delivery that completes the unit's tile count runs its tail
             if (tid == 0) s_last = (atomicAdd(&L.cnt[u].x, mine) + mine == total);
             __syncthreads();
-            if (s_last) {
+            if (s_last && !p.defer_tails) {
                 __threadfence();
                 constexpr int GB = G <= 4 ? 4 : 8;
                 TailPre<kSimtThreads, GB> pre;

@@ -43,13 +43,13 @@ def to_device(arr, torch, dtype, device):
 
 
 def make_context(w: Workload, kernel=mkv.MKV_KERNEL_AUTO, out_f32=True, sequences=None, record_probs=False,
-                 budget_max=None, layers=1):
+                 budget_max=None, layers=1, score_mode=mkv.MKV_SCORE_GROUP_MEAN):
     batch = w.batch if sequences is None else len(sequences)
     kv_dtype = mkv.MKV_BF16 if w.dtype == "bf16" else mkv.MKV_F32
     out_dtype = mkv.MKV_F32 if (out_f32 or kv_dtype == mkv.MKV_F32) else mkv.MKV_BF16
     lens = w.prefill_lens() if sequences is None else w.prefill_lens()[list(sequences)]
     return mkv.MomentKV(layers, w.q_heads, w.kv_heads, w.head_dim, budget_max or w.budget, w.beta, batch,
-                        int(max(lens.max(), 1)), kv_dtype=kv_dtype, out_dtype=out_dtype, kernel=kernel,
+                        int(max(lens.max(), 1)), kv_dtype=kv_dtype, out_dtype=out_dtype, kernel=kernel, score_mode=score_mode,
                         flags=mkv.MKV_FLAG_RECORD_PROBS if record_probs else 0)
 
 

@@ -207,3 +207,32 @@ def test_headline_shape_sampled_units_at_steady_state():
         want = g_pos[O.select(g_sc, g_pos, 1)]            # integer selection on the GPU's own scores
         assert want.tolist() == ev_pos.tolist()
     ctx.close()
+
+
+@pytest.mark.parametrize("shape", ["llama_bf16", "small_f32"])
+def test_layer_mean_mode_scores_over_all_heads(shape):
+    """MKV_SCORE_LAYER_MEAN with several KV heads (Eq. 4 as printed: the mean runs over all H
+    heads, one importance vector per sequence, every KV head evicts the same tokens)."""
+    from oracle import mkv_oracle as O
+    if shape == "llama_bf16":
+        w = CONFIGS["llama_b1"].with_(batch=2, prefill=(100, 300), steps=220, budget=90, variant="hot", n_heavy=3)
+    else:
+        w = CONFIGS["tiny"].with_(q_heads=6, kv_heads=2, batch=2, prefill=70, steps=200, budget=48, variant="hot")
+    ctx = make_context(w, score_mode=mkv.MKV_SCORE_LAYER_MEAN)
+    stream = BatchStream(w, 0)
+    oracles, _ = prefill_both(ctx, w, stream, mode=O.LAYER_MEAN)
+    rep = lockstep(ctx, w, stream, oracles, 150)
+    ctx.set_budget(w.budget - 20)                   # one step with overflow > 1 as well
+    for o in oracles:
+        o.set_budget(w.budget - 20)
+    rep = lockstep(ctx, w, stream, oracles, w.steps - 150, report=rep)
+    for b in range(w.batch):
+        ref_pos, ref_sc = ctx.decode_state(0, b, 0)
+        for g in range(1, w.kv_heads):               # identical token sets and scores in every KV head
+            pos, sc = ctx.decode_state(0, b, g)
+            np.testing.assert_array_equal(pos, ref_pos)
+            np.testing.assert_array_equal(sc, ref_sc)
+    ctx.close()
+    assert rep.ok(), rep.failures[:5]
+    assert rep.max_out_err <= (2e-3 if w.dtype == "bf16" else 1e-5) and rep.max_score_err <= 1e-4
+    assert rep.evicted_not_newest > 20
