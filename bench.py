@@ -254,7 +254,7 @@ def job_tokens_per_s(batch, steps, world, ms_max):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--steps", type=int, default=10000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="mkv", choices=["mkv", "reference"])
     ap.add_argument("--config", default="llama_b16", choices=sorted(CONFIGS))
