@@ -361,7 +361,15 @@ def main():
     # end to end through the host-buffer entry point: H2D of q,k,v and D2H of out every step
     e2e = None
     if not args.no_e2e:
-        hq, hk, hv = qs.cpu().pin_memory(), ks.cpu().pin_memory(), vs.cpu().pin_memory()
+        # one pinned buffer per step holding q | k_new | v_new back to back (a single H2D copy)
+        nq, nk = qs[0].numel(), ks[0].numel()
+        packed = torch.empty((ring, nq + 2 * nk), dtype=tdt).pin_memory()
+        packed[:, :nq] = qs.reshape(ring, -1).cpu()
+        packed[:, nq:nq + nk] = ks.reshape(ring, -1).cpu()
+        packed[:, nq + nk:] = vs.reshape(ring, -1).cpu()
+        hq = [packed[i, :nq] for i in range(ring)]
+        hk = [packed[i, nq:nq + nk] for i in range(ring)]
+        hv = [packed[i, nq + nk:] for i in range(ring)]
         hout = torch.empty((B, Hq, d), dtype=tdt).pin_memory()
         n_e2e = max(100, args.steps // 4)
         for i in range(10):

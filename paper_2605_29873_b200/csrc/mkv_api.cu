@@ -435,9 +435,18 @@ mkv_status mkv_decode_step_host(mkv_ctx* c, int layer, const void* qh, const voi
     const size_t nq = (size_t)c->batch * c->q_heads * c->head_dim, nk = (size_t)c->batch * c->kv_heads * c->head_dim;
     uint8_t *dq = c->ws + c->lay.stage_q, *dk = c->ws + c->lay.stage_k, *dv = c->ws + c->lay.stage_v,
             *dout = c->ws + c->lay.stage_out;
-    if (cudaMemcpyAsync(dq, qh, nq * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return MKV_ERR_CUDA;
-    if (cudaMemcpyAsync(dk, kh, nk * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return MKV_ERR_CUDA;
-    if (cudaMemcpyAsync(dv, vh, nk * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return MKV_ERR_CUDA;
+    const uint8_t* q8 = (const uint8_t*)qh;
+    if ((const uint8_t*)kh == q8 + nq * es && (const uint8_t*)vh == q8 + (nq + nk) * es) {
+        // q, k_new and v_new lie back to back on the host: one copy instead of three (the three
+        // staging regions are adjacent and at least as large)
+        dk = dq + nq * es;
+        dv = dk + nk * es;
+        if (cudaMemcpyAsync(dq, qh, (nq + 2 * nk) * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return MKV_ERR_CUDA;
+    } else {
+        if (cudaMemcpyAsync(dq, qh, nq * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return MKV_ERR_CUDA;
+        if (cudaMemcpyAsync(dk, kh, nk * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return MKV_ERR_CUDA;
+        if (cudaMemcpyAsync(dv, vh, nk * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return MKV_ERR_CUDA;
+    }
     const Params p = make_params(c, layer, dq, dk, dv, dout, kModeDecode);
     const mkv_status s = launch_step(c, layer, p, st);
     if (s != MKV_OK) return s;

@@ -85,7 +85,8 @@ def test_empty_prefill_and_bf16_out_through_host_api():
     ctx = make_context(w, out_f32=False)
     stream = BatchStream(w, 0)
     oracles, _ = prefill_both(ctx, w, stream)
-    rep = lockstep(ctx, w, stream, oracles, w.steps, host_api=True)
+    rep = lockstep(ctx, w, stream, oracles, 100, host_api=True)
+    rep = lockstep(ctx, w, stream, oracles, w.steps - 100, host_api=True, host_packed=True, report=rep)
     ctx.close()
     assert rep.ok(), rep.failures[:5]
     assert rep.evictions == (w.steps - w.budget) * w.kv_heads
