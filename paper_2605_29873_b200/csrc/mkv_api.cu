@@ -23,7 +23,7 @@ inline int elem_size(int dt) { return dt == MKV_BF16 ? 2 : 4; }
 
 struct LayerOff {
     size_t Kp, Vp, Kd, Vd, score, pos, n_dec, abar, n_prev, ev_k, ev_pos, ev_score, cta_unit0, cta_head0,
-        cta_headn, unit_lp, unit_next0, next, cnt, unit_step, end;
+        cta_headn, unit_lp, unit_next0, next, cnt, unit_step, seq_ticket, end;
 };
 // Scratch that lives for one step only, shared by all layers of the context (calls on a
 // context are ordered on one stream, and a step touches it only after every earlier kernel
@@ -90,6 +90,7 @@ bool make_layout(int layers, int batch, int q_heads, int kv_heads, int head_dim,
     L.lo.next = take(2 * U * 4);      // two copies each, alternating from launch to launch
     L.lo.cnt = take(2 * U * 8);
     L.lo.unit_step = take(U * 4);
+    L.lo.seq_ticket = take((size_t)batch * 4);
     L.lo.end = o;
     L.layer_bytes = o;
     L.total = L.layer0 + L.layer_bytes * (size_t)layers;
@@ -211,6 +212,7 @@ LayerDev layer_dev(const mkv_ctx* c, int layer) {
     d.part_o = (float*)(sb + so.part_o);
     d.part_ml = (float*)(sb + so.part_ml);
     d.unit_step = (int32_t*)(base + o.unit_step);
+    d.seq_ticket = (int32_t*)(base + o.seq_ticket);
     d.keys = (unsigned long long*)(sb + so.keys);
     d.list_a = (int32_t*)(sb + so.list_a);
     d.list_b = (int32_t*)(sb + so.list_b);
@@ -396,6 +398,7 @@ mkv_status mkv_prefill(mkv_ctx* c, int layer, const void* K, const void* V, cons
     ok &= cudaMemsetAsync(base + L.lo.n_prev, 0, U * 4, st) == cudaSuccess;
     ok &= cudaMemsetAsync(base + L.lo.ev_k, 0, U * 4, st) == cudaSuccess;
     ok &= cudaMemsetAsync(base + L.lo.unit_step, 0, U * 4, st) == cudaSuccess;
+    ok &= cudaMemsetAsync(base + L.lo.seq_ticket, 0, (size_t)c->batch * 4, st) == cudaSuccess;
     if (!ok) return MKV_ERR_CUDA;
     // host vectors above are pageable: the runtime has staged them before returning
     if (maxlen > 0) {

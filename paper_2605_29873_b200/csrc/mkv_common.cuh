@@ -78,6 +78,7 @@ struct LayerDev {
     float* part_o;     // [units][kMaxParts][G][d]
     float* part_ml;    // [units][kMaxParts][G][2]  (running max in log2 units, running sum)
     int32_t* unit_step;// [units] decode steps completed
+    int32_t* seq_ticket;  // [batch] KV heads of a sequence done (layer-wide score mode), zero between steps
     unsigned long long* keys;   // [units][cap] selection scratch
     int32_t* list_a;   // [units][cap] compaction scratch (holes)
     int32_t* list_b;   // [units][cap] compaction scratch (movers)

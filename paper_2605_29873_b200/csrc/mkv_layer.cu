@@ -1,10 +1,13 @@
 // Scoring exactly as Eq. 4 prints it: the attention a decode token receives is averaged over
 // ALL H query heads of the layer, the layer keeps ONE importance vector per sequence, and all
 // KV heads evict the same tokens (score mode MKV_SCORE_LAYER_MEAN with more than one KV
-// head).  The streaming kernels run unchanged but leave the unit tails out; this kernel, one
-// CTA per sequence, then does for all KV heads of the sequence what a unit tail does for one:
+// head).  The streaming kernels run unchanged but leave the unit tails out; this kernel then
+// does for all KV heads of a sequence what a unit tail does for one.  One CTA per
+// (sequence, KV head) handles that head's share; the CTA that finishes last for a sequence
+// (a ticket) does the part that needs all heads:
 //   per KV head: the fresh token's logits, the cross-split combine, `out`          (Eq. 2)
-//   per decode token: abar = (1/H) sum over all heads of 2^(s - M_h) / L_h           (Eq. 4)
+//                and, per decode token, the sum over its G heads of 2^(s - M_h) / L_h
+//   per decode token: abar = (1/H) sum of those sums over the KV heads               (Eq. 4)
 //   I <- beta * I + abar, the fresh token starting from 0                            (Eq. 5, 6)
 //   one selection of the overflow-many lowest (score bits, position id) keys         (Eq. 7, 8)
 //   the same append / hole filling in every KV head's pool                           (Eq. 9)
@@ -34,14 +37,16 @@ __global__ void __launch_bounds__(kLtThreads) layer_tail_kernel(const Params p) 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int G = p.group, D = p.head_dim, cap = p.cap, ls = p.lstride, Hkv = p.kv_heads, Hq = p.q_heads;
     const int rowb = D * (int)sizeof(T);
-    const int b = blockIdx.x, u0 = b * Hkv;
+    const int b = blockIdx.x / Hkv, u0 = b * Hkv;
     const int n_old = min(L.n_dec[u0], cap - 1);
     const int n = n_old + 1;
     const int t = L.unit_step[u0];
     const int k = max(0, n - p.budget);
+    __shared__ int s_last;
 
-    // ---- per KV head: fresh logits, combine, out ------------------------------------------------
-    for (int g = 0; g < Hkv; ++g) {
+    // ---- this CTA's KV head: fresh logits, combine, out, and its heads' share of Eq. 4 ------------
+    {
+        const int g = blockIdx.x - b * Hkv;
         const int u = u0 + g;
         const int P = min(__ldcg(&L.cnt[u].y), kMaxParts), part0 = u * kMaxParts;
         const T* qrow = reinterpret_cast<const T*>(p.q) + ((size_t)b * Hq + (size_t)g * G) * D;
@@ -90,24 +95,46 @@ __global__ void __launch_bounds__(kLtThreads) layer_tail_kernel(const Params p) 
             if (p.out_f32) reinterpret_cast<float*>(p.out)[obase + idx] = acc;
             else reinterpret_cast<__nv_bfloat16*>(p.out)[obase + idx] = __float2bfloat16_rn(acc);
         }
+        // sum over this KV head's G query heads of the normalised probabilities, per decode token
+        // (the fresh token last), parked in the unit's row of the compaction scratch
+        float* part = reinterpret_cast<float*>(L.list_b + (size_t)u * cap);
+        const float* lgu = L.logit + ((size_t)b * Hq + (size_t)g * G) * ls;
+        for (int i = tid; i < n_old; i += kLtThreads) {
+            float s = 0.f;
+            for (int h = 0; h < G; ++h) s = fmaf(fast_exp2(__ldcg(&lgu[(size_t)h * ls + i]) - sM[g * G + h]), sInvL[g * G + h], s);
+            part[i] = s;
+        }
+        if (tid == 0) {
+            float s = 0.f;
+            for (int h = 0; h < G; ++h) s = fmaf(sWnew[g * G + h], sInvL[g * G + h], s);
+            part[n_old] = s;
+        }
+        __threadfence();
         __syncthreads();
     }
+    // The CTA that finishes last for the sequence goes on (and leaves the ticket at zero).
+    if (tid == 0) {
+        s_last = (atomicAdd(&L.seq_ticket[b], 1) == Hkv - 1);
+        if (s_last) L.seq_ticket[b] = 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
 
-    // ---- probabilities over all heads, head mean, momentum update -------------------------------
+    // ---- all heads: head mean, momentum update -----------------------------------------------
     const float inv_h = 1.0f / (float)Hq;
     float ab_new = 0.f;
-    for (int h = 0; h < Hq; ++h) ab_new += sWnew[h] * sInvL[h];
+    for (int g = 0; g < Hkv; ++g) ab_new += __ldcg(reinterpret_cast<const float*>(L.list_b + (size_t)(u0 + g) * cap) + n_old);
     ab_new *= inv_h;                                   // Eq. 6: I_fresh = alpha * 0 + abar_fresh
     const unsigned long long key_new = ((unsigned long long)__float_as_uint(ab_new) << 32) | (unsigned)t;
     unsigned long long* keys = L.keys + (size_t)u0 * cap;
-    const float* lg = L.logit + (size_t)b * Hq * ls;
     const float* score0 = L.score + (size_t)u0 * ls;
     const int32_t* pos0 = L.pos + (size_t)u0 * ls;
     unsigned long long best_key = ~0ull;
     int best_slot = -1;
     for (int i = tid; i < n_old; i += kLtThreads) {
         float s = 0.f;
-        for (int h = 0; h < Hq; ++h) s = fmaf(fast_exp2(__ldcg(&lg[(size_t)h * ls + i]) - sM[h]), sInvL[h], s);
+        for (int g = 0; g < Hkv; ++g) s += __ldcg(reinterpret_cast<const float*>(L.list_b + (size_t)(u0 + g) * cap) + i);
         const float ab = s * inv_h;
         const float nw = fmaf(p.beta, score0[i], ab);
         for (int g = 0; g < Hkv; ++g) {
@@ -250,8 +277,9 @@ __global__ void __launch_bounds__(kLtThreads) layer_tail_kernel(const Params p) 
 bool layer_tail_supported(int q_heads, int group) { return q_heads <= kLtMaxHeads && group <= kMaxGroup; }
 
 cudaError_t launch_layer_tail(const Params& p, int kv_dtype, cudaStream_t st) {
-    if (kv_dtype == 0) layer_tail_kernel<__nv_bfloat16><<<p.batch, kLtThreads, 0, st>>>(p);
-    else layer_tail_kernel<float><<<p.batch, kLtThreads, 0, st>>>(p);
+    const unsigned grid = (unsigned)(p.batch * p.kv_heads);
+    if (kv_dtype == 0) layer_tail_kernel<__nv_bfloat16><<<grid, kLtThreads, 0, st>>>(p);
+    else layer_tail_kernel<float><<<grid, kLtThreads, 0, st>>>(p);
     return cudaGetLastError();
 }
 
