@@ -235,6 +235,7 @@ Params make_params(const mkv_ctx* c, int layer, const void* q, const void* k_new
     // Eq. 4 over all heads of the layer needs every KV head of a sequence: a second kernel
     p.defer_tails = (mode == kModeDecode && c->score_mode == MKV_SCORE_LAYER_MEAN && c->kv_heads > 1) ? 1 : 0;
     p.out_f32 = (c->out_dtype == MKV_F32);
+    p.launch_parity = (int)(c->launches & 1);
     return p;
 }
 

@@ -99,6 +99,7 @@ struct Params {
     int mode;
     int out_f32;
     int defer_tails;   // the unit tails are left to a following kernel (layer-wide score mode)
+    int launch_parity; // launches of the context so far, modulo 2 (diagnostic builds keep two trace sets)
 };
 
 // byte offset inside a stored row of logical byte `byte` for the row in slot `slot`
@@ -127,17 +128,19 @@ __device__ inline int unit_tiles(int lp, int n_old) {
 __device__ inline int unit_chunk(int total) { return max(2, (total + kMaxParts - 9) / (kMaxParts - 8)); }
 
 // Optional per-CTA timestamps (diagnostic builds only: compile with -DMKV_TRACE).  Slot i of
-// CTA c is g_trace[c * 16 + i]; mkv_debug_trace() copies the array to the host.
+// CTA c is g_trace[(launch parity * kMaxCtas + c) * 16 + i]; mkv_debug_trace() copies the array
+// to the host.
 #ifdef MKV_TRACE
-static __device__ unsigned long long g_trace[kMaxCtas * 16];   // one copy per translation unit
+static __device__ unsigned long long g_trace[2 * kMaxCtas * 16];   // one copy per translation unit
 __device__ inline unsigned long long trace_now() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-#define MKV_TR(i) (mkv::g_trace[blockIdx.x * 16 + (i)] = mkv::trace_now())
-#define MKV_TR_ADD(i, v) (mkv::g_trace[blockIdx.x * 16 + (i)] += (v))
-#define MKV_TR_SET(i, v) (mkv::g_trace[blockIdx.x * 16 + (i)] = (v))
+#define MKV_TR_AT(i) mkv::g_trace[(p.launch_parity * mkv::kMaxCtas + blockIdx.x) * 16 + (i)]
+#define MKV_TR(i) (MKV_TR_AT(i) = mkv::trace_now())
+#define MKV_TR_ADD(i, v) (MKV_TR_AT(i) += (v))
+#define MKV_TR_SET(i, v) (MKV_TR_AT(i) = (v))
 #else
 #define MKV_TR(i) ((void)0)
 #define MKV_TR_ADD(i, v) ((void)0)

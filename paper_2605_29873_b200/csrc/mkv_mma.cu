@@ -265,6 +265,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             }
         }
         ptx::griddep_wait();
+        if (lane == 0) MKV_TR(7);
         int n_old = min(L.n_dec[u], p.cap - (dec ? 1 : 0));
         int total = unit_tiles(lp, n_old);
         int chunk = unit_chunk(total);

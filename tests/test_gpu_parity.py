@@ -237,3 +237,40 @@ def test_layer_mean_mode_scores_over_all_heads(shape):
     assert rep.ok(), rep.failures[:5]
     assert rep.max_out_err <= (2e-3 if w.dtype == "bf16" else 1e-5) and rep.max_score_err <= 1e-4
     assert rep.evicted_not_newest > 20
+
+
+def test_error_paths_return_status_codes():
+    """Misuse is answered with a status code on the host, never with a device fault."""
+    import torch
+    w = CONFIGS["llama_b1"].with_(prefill=100, budget=32)
+    ctx = make_context(w)
+    dev = ctx.device
+    q = torch.zeros((1, w.q_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+    kv = torch.zeros((1, w.kv_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+    out = torch.zeros((1, w.q_heads, w.head_dim), dtype=torch.float32, device=dev)
+    with pytest.raises(mkv.MkvError) as e:
+        ctx.decode_step(0, q, kv, kv, out)                       # before any prefill
+    assert e.value.code == 2
+    K = torch.zeros((1, w.kv_heads, 200, w.head_dim), dtype=torch.bfloat16, device=dev)
+    with pytest.raises(mkv.MkvError) as e:
+        ctx.prefill(0, K, K, np.array([150], dtype=np.int32))    # longer than max_prefill (100)
+    assert e.value.code == 3
+    with pytest.raises(mkv.MkvError) as e:
+        ctx.prefill(1, K, K, np.array([50], dtype=np.int32))     # no such layer
+    assert e.value.code == 1
+    ctx.prefill(0, K, K, np.array([100], dtype=np.int32))
+    with pytest.raises(mkv.MkvError) as e:
+        ctx.set_budget(33)                                       # above the budget given at creation
+    assert e.value.code == 3
+    flat = torch.zeros(q.numel() + 8, dtype=torch.bfloat16, device=dev)
+    with pytest.raises(mkv.MkvError) as e:
+        ctx.decode_step(0, flat[1:1 + q.numel()].view_as(q), kv, kv, out)    # 2-byte aligned query
+    assert e.value.code == 1
+    ctx.decode_step(0, q, kv, kv, out)                           # and the context still works
+    ctx.status_sync()
+    assert ctx.step_count(0) == 1
+    ctx.reset()
+    with pytest.raises(mkv.MkvError) as e:
+        ctx.attend_only(0, q, out)                               # reset: back to "not prefilled"
+    assert e.value.code == 2
+    ctx.close()
