@@ -274,3 +274,36 @@ def test_error_paths_return_status_codes():
         ctx.attend_only(0, q, out)                               # reset: back to "not prefilled"
     assert e.value.code == 2
     ctx.close()
+
+
+@pytest.mark.parametrize("mode", ["group", "layer"])
+def test_head_averaged_probabilities_match_eq4(mode):
+    """MKV_FLAG_RECORD_PROBS: the head-averaged attention of every decode token (Eq. 4), fresh
+    token included, read back after each step and compared with the oracle's, in both score
+    modes.  Their sum over the decode pool is at most 1 (the rest went to the prefill pool)."""
+    import torch
+    from oracle import mkv_oracle as O
+    w = CONFIGS["llama_b1"].with_(prefill=150, steps=90, budget=60, variant="hot", n_heavy=2)
+    smode = mkv.MKV_SCORE_LAYER_MEAN if mode == "layer" else mkv.MKV_SCORE_GROUP_MEAN
+    ctx = make_context(w, record_probs=True, score_mode=smode)
+    stream = BatchStream(w, 0)
+    oracles, _ = prefill_both(ctx, w, stream, mode=O.LAYER_MEAN if mode == "layer" else O.GROUP_MEAN)
+    dt = ctx.torch_kv_dtype()
+    out = torch.zeros((1, w.q_heads, w.head_dim), dtype=torch.float32, device=ctx.device)
+    qs, ks, vs = stream.next(w.steps)
+    worst = 0.0
+    for i in range(w.steps):
+        ctx.decode_step(0, *(torch.from_numpy(np.ascontiguousarray(a[i], dtype=np.float32)).to(ctx.device, dt)
+                             for a in (qs, ks, vs)), out)
+        oracles[0].attend_update(qs[i, 0], ks[i, 0], vs[i, 0])
+        for g in range(w.kv_heads):
+            got = ctx.last_probs(0, 0, g).astype(np.float64)          # slot order before this step's eviction
+            _, _, o_ab = oracles[0].decode_state(g)                   # oracle: insertion order, before evict()
+            assert len(got) == len(o_ab) and got.sum() <= 1.0 + 1e-5 and (got > 0).all()
+            # compare as multisets keyed by value order: slot order differs from insertion order
+            np.testing.assert_allclose(np.sort(got), np.sort(o_ab), rtol=2e-4, atol=1e-9)
+            worst = max(worst, float(np.abs(np.sort(got) - np.sort(o_ab)).max()))
+        # keep the oracle in step with the GPU's eviction choice
+        oracles[0].evict(force=[ctx.last_evicted(0, 0, g)[0].astype(np.int64) for g in range(w.kv_heads)])
+    ctx.close()
+    assert worst < 1e-4
