@@ -147,6 +147,18 @@ mkv_status mkv_prefill(mkv_ctx* ctx, int layer, const void* K, const void* V,
                        const int32_t* prefill_lens, int src_rows, void* stream);
 
 /*
+ * The same with one prompt length per (sequence, KV head) unit: the shape of a frozen pool
+ * that a per-head prefill compressor (SnapKV- or PyramidKV-like; Sec. 5.4 of the paper runs
+ * Moment-KV on top of such pools) has already thinned out.  The compressors themselves are
+ * not part of this library: K and V hold, for unit (b, g), its retained rows first.
+ *   unit_lens     host pointer, [batch * kv_heads]; unit (b, g) uses rows [0, unit_lens[b*kv_heads+g])
+ * Errors as mkv_prefill; UNSUPPORTED with MKV_SCORE_LAYER_MEAN and several KV heads unless
+ * the KV heads of a sequence have equal lengths.
+ */
+mkv_status mkv_prefill_units(mkv_ctx* ctx, int layer, const void* K, const void* V,
+                             const int32_t* unit_lens, int src_rows, void* stream);
+
+/*
  * One decode step of Algorithm 1 for one layer, all sequences:
  *   append (k_new, v_new) with importance 0; attention of q over prefill U decode pool
  *   (Eq. 2), fresh token included; per decode token the head-averaged probability

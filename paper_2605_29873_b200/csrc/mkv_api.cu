@@ -125,16 +125,16 @@ __global__ void prefill_copy_kernel(const uint8_t* __restrict__ srcK, const uint
 // unit has that many prefill tiles left to give (these can be fetched before the previous
 // step has finished); everything else is handed out by the unit's counter, which
 // therefore starts behind the reserved tiles.  Returns the number of CTAs (the grid).
-int build_start_table(int batch, int kv_heads, int budget, const int32_t* prefill_lens, int n_ctas_max,
+int build_start_table(int units, int budget, const int32_t* unit_lens, int n_ctas_max,
                       std::vector<int32_t>& lp, std::vector<int32_t>& next0, std::vector<int32_t>& cta_unit0,
                       std::vector<int32_t>& cta_head0, std::vector<int32_t>& cta_headn) {
-    const int U = batch * kv_heads;
+    const int U = units;
     const int td = ceil_div(budget, kTileRows);
     lp.assign(U, 0);
     next0.assign(U, 0);
     std::vector<long long> tile_begin(U + 1, 0);
     for (int u = 0; u < U; ++u) {
-        lp[u] = prefill_lens[u / kv_heads];
+        lp[u] = unit_lens[u];
         tile_begin[u + 1] = tile_begin[u] + ceil_div(lp[u], kTileRows) + td;
     }
     const long long t_all = tile_begin[U];
@@ -174,7 +174,7 @@ struct mkv_ctx {
     bool pdl;
     std::vector<int> n_ctas;
     std::vector<int64_t> layer_launches;   // steps launched on a layer: its parity picks the counter copy
-    std::vector<std::vector<int32_t>> lens;   // per layer, per sequence
+    std::vector<std::vector<int32_t>> lens;   // per layer, per (sequence, KV head) unit
     int64_t launches;
 };
 
@@ -287,8 +287,9 @@ mkv_status mkv_plan_starts(int batch, int kv_heads, int budget, const int32_t* p
     if (!n_ctas || !cta_unit0 || !cta_head0 || !cta_headn || !unit_next0) return MKV_ERR_INVALID_ARG;
     for (int b = 0; b < batch; ++b)
         if (prefill_lens[b] < 0) return MKV_ERR_INVALID_ARG;
-    std::vector<int32_t> lp, next0, u0, h0, hn;
-    const int n = build_start_table(batch, kv_heads, budget, prefill_lens, n_ctas_max, lp, next0, u0, h0, hn);
+    std::vector<int32_t> lp, next0, u0, h0, hn, ul((size_t)batch * kv_heads);
+    for (size_t u = 0; u < ul.size(); ++u) ul[u] = prefill_lens[u / kv_heads];
+    const int n = build_start_table(batch * kv_heads, budget, ul.data(), n_ctas_max, lp, next0, u0, h0, hn);
     *n_ctas = n;
     std::memcpy(cta_unit0, u0.data(), sizeof(int32_t) * (size_t)n);
     std::memcpy(cta_head0, h0.data(), sizeof(int32_t) * (size_t)n);
@@ -354,7 +355,7 @@ mkv_status mkv_create(int layers, int q_heads, int kv_heads, int head_dim, int b
     if (const char* e = std::getenv("MKV_NO_OVERLAP")) c->pdl = std::atoi(e) == 0;
     c->n_ctas.assign(layers, 0);
     c->layer_launches.assign(layers, 0);
-    c->lens.assign(layers, std::vector<int32_t>(batch, 0));
+    c->lens.assign(layers, std::vector<int32_t>((size_t)batch * kv_heads, 0));
     c->launches = 0;
     *out_ctx = c;
     return MKV_OK;
@@ -364,12 +365,25 @@ void mkv_destroy(mkv_ctx* ctx) { delete ctx; }
 
 mkv_status mkv_prefill(mkv_ctx* c, int layer, const void* K, const void* V, const int32_t* prefill_lens,
                        int src_rows, void* stream) {
-    if (!layer_ok(c, layer) || !prefill_lens || src_rows < 0) return MKV_ERR_INVALID_ARG;
+    if (!layer_ok(c, layer) || !prefill_lens) return MKV_ERR_INVALID_ARG;
+    std::vector<int32_t> ul((size_t)c->batch * c->kv_heads);
+    for (size_t u = 0; u < ul.size(); ++u) ul[u] = prefill_lens[u / c->kv_heads];
+    return mkv_prefill_units(c, layer, K, V, ul.data(), src_rows, stream);
+}
+
+mkv_status mkv_prefill_units(mkv_ctx* c, int layer, const void* K, const void* V, const int32_t* unit_lens,
+                             int src_rows, void* stream) {
+    if (!layer_ok(c, layer) || !unit_lens || src_rows < 0) return MKV_ERR_INVALID_ARG;
+    if (c->score_mode == MKV_SCORE_LAYER_MEAN && c->kv_heads > 1) {
+        // one importance vector per sequence only makes sense over equal prompts per KV head
+        for (int u = 0; u < c->lay.units; ++u)
+            if (unit_lens[u] != unit_lens[u - u % c->kv_heads]) return MKV_ERR_UNSUPPORTED;
+    }
     int maxlen = 0;
-    for (int b = 0; b < c->batch; ++b) {
-        if (prefill_lens[b] < 0 || prefill_lens[b] > src_rows) return MKV_ERR_INVALID_ARG;
-        if (prefill_lens[b] > c->max_prefill) return MKV_ERR_CAPACITY;
-        maxlen = std::max(maxlen, prefill_lens[b]);
+    for (int u = 0; u < c->lay.units; ++u) {
+        if (unit_lens[u] < 0 || unit_lens[u] > src_rows) return MKV_ERR_INVALID_ARG;
+        if (unit_lens[u] > c->max_prefill) return MKV_ERR_CAPACITY;
+        maxlen = std::max(maxlen, unit_lens[u]);
     }
     if (maxlen > 0 && (!K || !V)) return MKV_ERR_INVALID_ARG;
     DeviceGuard guard(c->device);
@@ -379,10 +393,10 @@ mkv_status mkv_prefill(mkv_ctx* c, int layer, const void* K, const void* V, cons
     const int U = L.units;
 
     std::vector<int32_t> lp, next0, cta_unit0, cta_head0, cta_headn;
-    const int n_ctas = build_start_table(c->batch, c->kv_heads, c->budget_max, prefill_lens, c->n_ctas_max, lp, next0,
+    const int n_ctas = build_start_table(U, c->budget_max, unit_lens, c->n_ctas_max, lp, next0,
                                          cta_unit0, cta_head0, cta_headn);
     c->n_ctas[layer] = n_ctas;
-    for (int b = 0; b < c->batch; ++b) c->lens[layer][b] = prefill_lens[b];
+    for (int u = 0; u < U; ++u) c->lens[layer][u] = unit_lens[u];
 
     uint8_t* base = c->ws + L.layer0 + L.layer_bytes * (size_t)layer;
     bool ok = true;
@@ -561,7 +575,7 @@ mkv_status mkv_read_kv(mkv_ctx* c, int layer, int b, int g, int pool, int32_t* n
     const int rowb = c->lay.rowb;
     int count;
     size_t base;
-    if (pool == 0) { count = c->lens[layer][b]; base = (size_t)u * c->max_prefill * rowb; }
+    if (pool == 0) { count = c->lens[layer][u]; base = (size_t)u * c->max_prefill * rowb; }
     else { MKV_D2H(&count, d.n_dec + u, 4); base = (size_t)u * c->lay.cap * rowb; }
     *n = count;
     const int rows = std::min(count, cap_tokens);

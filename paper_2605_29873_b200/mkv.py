@@ -21,7 +21,7 @@ EXPORTED_SYMBOLS = [
     "mkv_workspace_bytes", "mkv_kv_bytes_per_token", "mkv_create", "mkv_destroy", "mkv_prefill",
     "mkv_decode_step", "mkv_decode_step_host", "mkv_attend_only", "mkv_set_budget", "mkv_reset",
     "mkv_status_sync", "mkv_launch_count", "mkv_get_decode_state", "mkv_get_last_evicted",
-    "mkv_get_last_probs", "mkv_read_kv", "mkv_get_step", "mkv_status_string", "mkv_attend_noalloc", "mkv_plan_starts",
+    "mkv_get_last_probs", "mkv_read_kv", "mkv_get_step", "mkv_status_string", "mkv_attend_noalloc", "mkv_plan_starts", "mkv_prefill_units",
 ]
 
 
@@ -53,6 +53,7 @@ def load_library(path: str | None = None):
     L.mkv_destroy.restype = None
     L.mkv_destroy.argtypes = [vp]
     L.mkv_prefill.argtypes = [vp, C.c_int, vp, vp, i32p, C.c_int, vp]
+    L.mkv_prefill_units.argtypes = [vp, C.c_int, vp, vp, i32p, C.c_int, vp]
     L.mkv_decode_step.argtypes = [vp, C.c_int, vp, vp, vp, vp, vp]
     L.mkv_decode_step_host.argtypes = [vp, C.c_int, vp, vp, vp, vp, vp]
     L.mkv_attend_only.argtypes = [vp, C.c_int, vp, vp, vp]
@@ -197,6 +198,16 @@ class MomentKV:
             assert tuple(K.shape) == (self.batch, self.kv_heads, src_rows, self.head_dim) == tuple(V.shape)
         _check(self._L.mkv_prefill(self._ctx, layer, _ptr(K), _ptr(V), lens.ctypes.data_as(C.POINTER(C.c_int32)),
                                    src_rows, self._stream(stream)), "mkv_prefill")
+
+    def prefill_units(self, layer, K, V, unit_lens, stream=None):
+        """As prefill, with one length per (sequence, KV head): unit_lens [batch, kv_heads] ints."""
+        lens = np.ascontiguousarray(unit_lens, dtype=np.int32).reshape(-1)
+        assert lens.shape == (self.batch * self.kv_heads,)
+        src_rows = int(K.shape[2])
+        assert K.is_contiguous() and V.is_contiguous() and K.dtype == self.torch_kv_dtype()
+        assert tuple(K.shape) == (self.batch, self.kv_heads, src_rows, self.head_dim) == tuple(V.shape)
+        _check(self._L.mkv_prefill_units(self._ctx, layer, _ptr(K), _ptr(V), lens.ctypes.data_as(C.POINTER(C.c_int32)),
+                                         src_rows, self._stream(stream)), "mkv_prefill_units")
 
     def decode_step(self, layer, q, k_new, v_new, out, stream=None):
         _check(self._L.mkv_decode_step(self._ctx, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out),
