@@ -318,17 +318,20 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             int found = -1;
             for (int base = 1; base < U && found < 0; base += 32) {
                 const int k = base + lane;
-                int lpc = 0, ndc = 0;
-                bool has = false;
+                int lpc = 0, ndc = 0, rem = 0;
                 if (k < U) {
                     const int cand = (u + k) % U;
                     lpc = L.unit_lp[cand];
                     ndc = min(L.n_dec[cand], p.cap - (dec ? 1 : 0));
-                    has = __ldcg(&L.next[cand]) < unit_tiles(lpc, ndc);
+                    rem = max(0, unit_tiles(lpc, ndc) - __ldcg(&L.next[cand]));
                 }
-                const unsigned ballot = __ballot_sync(0xffffffffu, has);
-                if (ballot) {
-                    const int src = __ffs(ballot) - 1;
+                // of these 32 units take the one with the most tiles left (the nearest on a tie):
+                // help goes where a slow CTA has fallen behind, and fewer visits end after one chunk
+                int best = (rem << 5) | (31 - lane);
+#pragma unroll
+                for (int off = 16; off; off >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, off));
+                if (best >> 5) {
+                    const int src = 31 - (best & 31);
                     found = (u + base + src) % U;
                     lp = __shfl_sync(0xffffffffu, lpc, src);
                     n_old = __shfl_sync(0xffffffffu, ndc, src);
