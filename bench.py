@@ -265,6 +265,7 @@ def main():
     ap.add_argument("--budget", type=int, default=0, help="override the workload's decode budget (profiling small cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay timing")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -317,15 +318,24 @@ def main():
     def step(i):
         ctx.decode_step(i % args.layers, qs[i % ring], ks[i % ring], vs[i % ring], out)
 
-    # set-up, not warm-up: fill every layer's decode pool to the budget (steady state)
-    for i in range(w.budget * args.layers):
-        step(i)
+    stream = torch.cuda.current_stream(dev)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # The ramp: every layer's decode pool from empty to the budget, timed on its own (steps get
+    # longer as the pool grows); it also is the set-up of the steady state measured below.
+    # Plain attention launches warm the kernel up first: they leave the state alone.
+    for i in range(10):
+        ctx.attend_only(i % args.layers, qs[i % ring], out)
     torch.cuda.synchronize()
+    n_ramp = w.budget * args.layers
+    ev0.record(stream)
+    for i in range(n_ramp):
+        step(i)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    ms_ramp = ev0.elapsed_time(ev1) / n_ramp
     ctx.status_sync()
     for i in range(args.warmup):
         step(i)
-    stream = torch.cuda.current_stream(dev)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(local)
 
     def barrier():
@@ -358,6 +368,28 @@ def main():
     barrier()
     ms_att = ev0.elapsed_time(ev1) / n_att
 
+    # the same steps recorded once and replayed as a CUDA graph (what a serving loop would do):
+    # launch cost leaves the host, which shows on the small, launch-bound workloads
+    ms_graph, n_rec = 0.0, 16 * args.layers
+    if not args.no_graph:
+        side = torch.cuda.Stream(dev)
+        side.wait_stream(stream)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(n_rec):
+                step(i)
+        reps = max(3, args.steps // n_rec)
+        for _ in range(3):
+            graph.replay()
+        barrier()
+        ev0.record(stream)
+        for _ in range(reps):
+            graph.replay()
+        ev1.record(stream)
+        barrier()
+        ms_graph = ev0.elapsed_time(ev1) / (reps * n_rec)
+        ctx.status_sync()
+
     # end to end through the host-buffer entry point: H2D of q,k,v and D2H of out every step
     e2e = None
     if not args.no_e2e:
@@ -387,7 +419,8 @@ def main():
         e2e = {"ms": ms_e2e, "steps": n_e2e, "h2d": (qs[0].numel() + ks[0].numel() + vs[0].numel()) * es,
                "d2h": hout.numel() * hout.element_size()}
 
-    ms_max, ms_att_max, ms_e2e_max = max_over_ranks([ms, ms_att, e2e["ms"] / e2e["steps"] if e2e else 0.0], world, dev)
+    ms_max, ms_att_max, ms_e2e_max, ms_ramp_max, ms_graph_max = max_over_ranks(
+        [ms, ms_att, e2e["ms"] / e2e["steps"] if e2e else 0.0, ms_ramp, ms_graph], world, dev)
 
     if rank == 0:
         ms_per_step = ms_max / args.steps
@@ -411,6 +444,18 @@ def main():
                          "kernel": "mma_kernel" if ctx_uses_mma(args, w) else "simt_kernel"},
             "attend_only": {"ms_per_step": ms_att_max, "overhead_ratio": ms_per_step / ms_att_max},
         }
+        # whole run of the workload (its step count per layer): the measured ramp, then steady state
+        T = max(int(w.steps), 1)
+        fill = min(w.budget, T)
+        run_ms = ms_ramp_max * fill + ms_per_step * (T - fill)
+        line["ramp"] = {"ms_per_step": ms_ramp_max, "steps_per_layer": w.budget,
+                        "what": "decode pool from empty to the budget, mean over the fill"}
+        line["whole_run"] = {"steps_per_layer": T, "ms_per_step": run_ms / T,
+                             "tokens_per_s": world * B * T / (run_ms * 1e-3),
+                             "how": "measured ramp mean x fill steps + measured steady state x the rest"}
+        if ms_graph_max > 0.0:
+            line["graph_replay"] = {"ms_per_step": ms_graph_max, "steps_per_graph": n_rec,
+                                    "tokens_per_s": world * B / (ms_graph_max * 1e-3)}
         if e2e:
             line["e2e"] = {"value": world * B / (ms_e2e_max * 1e-3), "unit": "tokens/s",
                            "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],

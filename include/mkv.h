@@ -29,6 +29,14 @@
  *   - One host thread at a time per context, and all calls of a context on one stream (or
  *     ordered by the caller in some other way): the layers of a context share the per-step
  *     scratch, and a step may begin while the previous kernel of its stream is still ending.
+ *   - Stream capture: mkv_decode_step() and mkv_attend_only() only enqueue kernels, so a
+ *     sequence of them (any number, any layers) can be recorded into a CUDA graph and replayed
+ *     any number of times; step numbers, pool counts and the work-sharing state live on the
+ *     device (Algorithm 1 has no host-side state).  A recording holds the pointers, the budget
+ *     and the launch plan of the moment: record again after mkv_prefill*() or mkv_set_budget().
+ *     mkv_prefill*(), the *_host entry points and the mkv_get_*() readers synchronise or copy
+ *     from pageable memory and cannot be recorded.  mkv_launch_count() counts enqueued
+ *     kernels, not replays.
  */
 #ifndef MKV_H_
 #define MKV_H_

@@ -23,7 +23,7 @@ inline int elem_size(int dt) { return dt == MKV_BF16 ? 2 : 4; }
 
 struct LayerOff {
     size_t Kp, Vp, Kd, Vd, score, pos, n_dec, abar, n_prev, ev_k, ev_pos, ev_score, cta_unit0, cta_head0,
-        cta_headn, unit_lp, unit_next0, next, cnt, unit_step, seq_ticket, end;
+        cta_headn, unit_lp, unit_next0, next, cnt, launch_no, unit_step, seq_ticket, end;
 };
 // Scratch that lives for one step only, shared by all layers of the context (calls on a
 // context are ordered on one stream, and a step touches it only after every earlier kernel
@@ -89,6 +89,7 @@ bool make_layout(int layers, int batch, int q_heads, int kv_heads, int head_dim,
     L.lo.unit_next0 = take(U * 4);
     L.lo.next = take(2 * U * 4);      // two copies each, alternating from launch to launch
     L.lo.cnt = take(2 * U * 8);
+    L.lo.launch_no = take((size_t)kMaxCtas * 4);   // per CTA: launches since the prefill
     L.lo.unit_step = take(U * 4);
     L.lo.seq_ticket = take((size_t)batch * 4);
     L.lo.end = o;
@@ -173,7 +174,6 @@ struct mkv_ctx {
     std::vector<char> stepped;   // a step has run on the layer since its prefill
     bool pdl;
     std::vector<int> n_ctas;
-    std::vector<int64_t> layer_launches;   // steps launched on a layer: its parity picks the counter copy
     std::vector<std::vector<int32_t>> lens;   // per layer, per (sequence, KV head) unit
     int64_t launches;
 };
@@ -186,7 +186,6 @@ LayerDev layer_dev(const mkv_ctx* c, int layer) {
     const LayerOff& o = c->lay.lo;
     const ScratchOff& so = c->lay.so;
     const size_t U = (size_t)c->lay.units;
-    const size_t cur = (size_t)(c->layer_launches[layer] & 1), idle = cur ^ 1;
     LayerDev d;
     d.Kp = base + o.Kp; d.Vp = base + o.Vp; d.Kd = base + o.Kd; d.Vd = base + o.Vd;
     d.score = (float*)(base + o.score);
@@ -205,10 +204,9 @@ LayerDev layer_dev(const mkv_ctx* c, int layer) {
     d.cta_headn = (const int32_t*)(base + o.cta_headn);
     d.unit_lp = (const int32_t*)(base + o.unit_lp);
     d.unit_next0 = (const int32_t*)(base + o.unit_next0);
-    d.next = (int32_t*)(base + o.next) + cur * U;
-    d.cnt = (int2*)(base + o.cnt) + cur * U;
-    d.next_idle = (int32_t*)(base + o.next) + idle * U;
-    d.cnt_idle = (int2*)(base + o.cnt) + idle * U;
+    d.next = (int32_t*)(base + o.next);
+    d.cnt = (int2*)(base + o.cnt);
+    d.launch_no = (uint32_t*)(base + o.launch_no);
     d.part_o = (float*)(sb + so.part_o);
     d.part_ml = (float*)(sb + so.part_ml);
     d.unit_step = (int32_t*)(base + o.unit_step);
@@ -250,7 +248,6 @@ mkv_status launch_step(mkv_ctx* c, int layer, const Params& p, cudaStream_t st) 
         if (launch_layer_tail(p, c->kv_dtype, st) != cudaSuccess) return MKV_ERR_CUDA;
         c->launches += 1;
     }
-    c->layer_launches[layer] += 1;
     c->stepped[layer] = 1;
     return MKV_OK;
 }
@@ -354,7 +351,6 @@ mkv_status mkv_create(int layers, int q_heads, int kv_heads, int head_dim, int b
     c->pdl = true;
     if (const char* e = std::getenv("MKV_NO_OVERLAP")) c->pdl = std::atoi(e) == 0;
     c->n_ctas.assign(layers, 0);
-    c->layer_launches.assign(layers, 0);
     c->lens.assign(layers, std::vector<int32_t>((size_t)batch * kv_heads, 0));
     c->launches = 0;
     *out_ctx = c;
@@ -408,6 +404,7 @@ mkv_status mkv_prefill_units(mkv_ctx* c, int layer, const void* K, const void* V
     ok &= cudaMemcpyAsync(base + L.lo.next, next0.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok &= cudaMemcpyAsync(base + L.lo.next + (size_t)U * 4, next0.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok &= cudaMemsetAsync(base + L.lo.cnt, 0, 2 * (size_t)U * 8, st) == cudaSuccess;
+    ok &= cudaMemsetAsync(base + L.lo.launch_no, 0, (size_t)kMaxCtas * 4, st) == cudaSuccess;
     // empty decode pool, rewind counters
     ok &= cudaMemsetAsync(base + L.lo.n_dec, 0, U * 4, st) == cudaSuccess;
     ok &= cudaMemsetAsync(base + L.lo.n_prev, 0, U * 4, st) == cudaSuccess;

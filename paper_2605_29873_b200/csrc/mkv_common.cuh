@@ -71,10 +71,14 @@ struct LayerDev {
     const int32_t* cta_headn;   // [n_ctas] number of reserved tiles (prefill tiles; may be 0)
     const int32_t* unit_lp;     // [units] prefill length
     const int32_t* unit_next0;  // [units] tiles reserved in the unit = start value of its counter
-    int32_t* next;     // [units] tiles handed out so far (this launch's copy)
-    int2* cnt;         // [units] x: tiles delivered so far, y: partial slots taken so far
-    int32_t* next_idle;   // the other copies, rewound by the tails for the next launch
-    int2* cnt_idle;
+    // Work-sharing counters, two copies each (copy c at + c * n_units).  A launch uses the copy
+    // of its own parity and its tails rewind the other one for the launch after it.  The parity
+    // is found on the device: every CTA keeps, in a word of its own, the number of launches it
+    // has taken part in since the layer's prefill (the grid does not change in between) -- so
+    // a recorded sequence of launches (a CUDA graph) can be replayed any number of times.
+    int32_t* next;     // [2][units] tiles handed out so far
+    int2* cnt;         // [2][units] x: tiles delivered so far, y: partial slots taken so far
+    uint32_t* launch_no;   // [kMaxCtas] launches CTA i has taken part in since the layer's prefill
     float* part_o;     // [units][kMaxParts][G][d]
     float* part_ml;    // [units][kMaxParts][G][2]  (running max in log2 units, running sum)
     int32_t* unit_step;// [units] decode steps completed
@@ -101,6 +105,15 @@ struct Params {
     int defer_tails;   // the unit tails are left to a following kernel (layer-wide score mode)
     int launch_parity; // launches of the context so far, modulo 2 (diagnostic builds keep two trace sets)
 };
+
+// Parity of the launch this CTA is part of; counts the launch in the CTA's own word.  Call once
+// per CTA, from one thread, after every earlier kernel of the stream has completed.  (The
+// tensor-core kernel does the same by hand, with other work between the load and its use.)
+__device__ inline int take_launch_parity(const LayerDev& L) {
+    const uint32_t v = __ldcg(&L.launch_no[blockIdx.x]);
+    L.launch_no[blockIdx.x] = v + 1u;
+    return (int)(v & 1u);
+}
 
 // byte offset inside a stored row of logical byte `byte` for the row in slot `slot`
 __host__ __device__ inline uint32_t swz(uint32_t slot, uint32_t byte) {

@@ -43,12 +43,15 @@ __global__ void __launch_bounds__(kLtThreads) layer_tail_kernel(const Params p) 
     const int t = L.unit_step[u0];
     const int k = max(0, n - p.budget);
     __shared__ int s_last;
+    // the streaming kernel of this step has finished and has counted itself: its parity is
+    // that of the launch before the count now stored
+    const int par = (int)((__ldcg(&L.launch_no[0]) & 1u) ^ 1u);
 
     // ---- this CTA's KV head: fresh logits, combine, out, and its heads' share of Eq. 4 ------------
     {
         const int g = blockIdx.x - b * Hkv;
         const int u = u0 + g;
-        const int P = min(__ldcg(&L.cnt[u].y), kMaxParts), part0 = u * kMaxParts;
+        const int P = min(__ldcg(&L.cnt[(size_t)par * L.n_units + u].y), kMaxParts), part0 = u * kMaxParts;
         const T* qrow = reinterpret_cast<const T*>(p.q) + ((size_t)b * Hq + (size_t)g * G) * D;
         const T* knew = reinterpret_cast<const T*>(p.k_new) + (size_t)u * D;
         const T* vnew = reinterpret_cast<const T*>(p.v_new) + (size_t)u * D;
@@ -153,7 +156,7 @@ __global__ void __launch_bounds__(kLtThreads) layer_tail_kernel(const Params p) 
     if (tid < Hkv) {
         const int u = u0 + tid;
         L.n_prev[u] = n; L.ev_k[u] = k; L.n_dec[u] = n - k; L.unit_step[u] = t + 1;
-        rewind_unit(L, u);
+        rewind_unit(L, u, par);
     }
 
     // the fresh row of KV head g into slot `dst` of its pool, with the shared score and id

@@ -87,6 +87,7 @@ struct Control {
     ExchangeRef xq[kMaxStages];
     int abort_flag;
     int tail_unit;     // partial slots of the unit whose tail is due, or -1
+    int par;           // parity of this launch (the producer finds it after the dependency wait); -1 before
 };
 
 constexpr size_t smem_bytes(int nst) {
@@ -128,8 +129,16 @@ __device__ void tail_group(const Params& p, Control* ctl, TailSmem<kTailThreads>
             const int total = unit_tiles(L.unit_lp[u], min(pre.n_dec, p.cap - (dec ? 1 : 0)));
             const unsigned long long t0 = ptx::globaltimer_ns();
             int slots = -1;
-            for (;;) {
-                const unsigned long long w = *reinterpret_cast<const volatile unsigned long long*>(&L.cnt[u]);
+            int par = tsm->par;
+            while (par < 0) {   // first unit: the producer has not read the launch's parity yet
+                par = *reinterpret_cast<const volatile int*>(&ctl->par);
+                if (par >= 0) { tsm->par = par; break; }
+                if (aborted(ctl)) break;
+                if (ptx::globaltimer_ns() - t0 > kWaitNs) { note_timeout(p, ctl); break; }
+            }
+            const int2* cnt_u = L.cnt + (size_t)max(par, 0) * L.n_units + u;
+            for (; par >= 0;) {
+                const unsigned long long w = *reinterpret_cast<const volatile unsigned long long*>(cnt_u);
                 if ((int)(unsigned)(w & 0xffffffffull) >= total) { slots = (int)(unsigned)(w >> 32); break; }
                 if (aborted(ctl)) break;
                 if (ptx::globaltimer_ns() - t0 > kWaitNs) { note_timeout(p, ctl); break; }
@@ -173,6 +182,8 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         }
         ctl->abort_flag = 0;
         ctl->tail_unit = -1;
+        ctl->par = -1;
+        tsm->par = -1;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async();
     }
@@ -266,28 +277,46 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         }
         ptx::griddep_wait();
         if (lane == 0) MKV_TR(7);
-        int n_old = min(L.n_dec[u], p.cap - (dec ? 1 : 0));
-        int total = unit_tiles(lp, n_old);
-        int chunk = unit_chunk(total);
-        if (lane == 0 && ok && head_end > L.cta_head0[blockIdx.x]) {
-            slot = atomicAdd(&L.cnt[u].y, 1);
+        // Loads first, then the query copy, then their use: the consumers wait for the query, which
+        // must not wait for a load's round trip.
+        int n_old = L.n_dec[u];
+        uint32_t seen = 0;         // launches this CTA has taken part in (lane 0)
+        if (lane == 0) seen = __ldcg(&L.launch_no[blockIdx.x]);
+        const bool has_head = head_end > L.cta_head0[blockIdx.x];
+        if (lane == 0 && ok && has_head) {
             ok = issue_query(u);
             q_sent = true;
+        }
+        n_old = min(n_old, p.cap - (dec ? 1 : 0));
+        // which copy of the unit counters this launch uses
+        int par = 0;
+        if (lane == 0) {
+            par = (int)(seen & 1u);
+            L.launch_no[blockIdx.x] = seen + 1u;
+            *reinterpret_cast<volatile int*>(&ctl->par) = par;
+        }
+        par = __shfl_sync(0xffffffffu, par, 0);
+        int32_t* const nxt = L.next + (size_t)par * L.n_units;
+        int2* const cnt = L.cnt + (size_t)par * L.n_units;
+        int total = unit_tiles(lp, n_old);
+        int chunk = unit_chunk(total);
+        if (lane == 0 && ok && has_head) {
+            slot = atomicAdd(&cnt[u].y, 1);
             for (; head_t < head_end && ok; ++head_t) {
                 ok = issue_tile(u, tile_ref(head_t, lp, 0), sent == 0);
                 ++sent; ++mine;
             }
         }
         int g = 0;                 // first tile of the chunk in hand
-        if (lane == 0) g = atomicAdd(&L.next[u], chunk);
+        if (lane == 0) g = atomicAdd(&nxt[u], chunk);
         for (;;) {
             g = __shfl_sync(0xffffffffu, g, 0);
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
             if (g < total) {
                 if (lane == 0) {
-                    const int g_next = atomicAdd(&L.next[u], chunk);   // in flight while this chunk is issued
-                    if (slot < 0) slot = atomicAdd(&L.cnt[u].y, 1);
+                    const int g_next = atomicAdd(&nxt[u], chunk);   // in flight while this chunk is issued
+                    if (slot < 0) slot = atomicAdd(&cnt[u].y, 1);
                     const int t_end = min(g + chunk, total);
                     for (int t = g; t < t_end && ok; ++t) {
                         const TileRef tr = tile_ref(t, lp, n_old);
@@ -323,7 +352,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
                     const int cand = (u + k) % U;
                     lpc = L.unit_lp[cand];
                     ndc = min(L.n_dec[cand], p.cap - (dec ? 1 : 0));
-                    rem = max(0, unit_tiles(lpc, ndc) - __ldcg(&L.next[cand]));
+                    rem = max(0, unit_tiles(lpc, ndc) - __ldcg(&nxt[cand]));
                 }
                 // of these 32 units take the one with the most tiles left (the nearest on a tie):
                 // help goes where a slow CTA has fallen behind, and fewer visits end after one chunk
@@ -341,7 +370,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             u = found;
             total = unit_tiles(lp, n_old);
             chunk = unit_chunk(total);
-            if (lane == 0) g = atomicAdd(&L.next[u], chunk);
+            if (lane == 0) g = atomicAdd(&nxt[u], chunk);
         }
         if (lane == 0) {
             if (ok && acquire()) {
@@ -565,7 +594,12 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             __threadfence();
             __syncwarp();
             // The tail group that looks after this unit watches the count; nothing to announce.
-            if (lane == 0) { MKV_TR(4); atomicAdd(&L.cnt[u].x, ref.ntiles); }
+            if (lane == 0) {
+                MKV_TR(4);
+                // (the producer wrote the parity before it sent this visit's first counter pull)
+                const int par = *reinterpret_cast<const volatile int*>(&ctl->par);
+                atomicAdd(&L.cnt[(size_t)par * L.n_units + u].x, ref.ntiles);
+            }
         }
     } else {
         // ================================ tail warps ===================================

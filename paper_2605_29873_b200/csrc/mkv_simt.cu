@@ -56,6 +56,12 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
     const int U = L.n_units;
     __shared__ int s_g, s_u;
 
+    // which copy of the unit counters this launch uses
+    if (tid == 0) tsm.par = take_launch_parity(L);
+    __syncthreads();
+    int32_t* const nxt = L.next + (size_t)tsm.par * L.n_units;
+    int2* const cnt = L.cnt + (size_t)tsm.par * L.n_units;
+
     int u = L.cta_unit0[blockIdx.x];
     int head = L.cta_head0[blockIdx.x], headn = L.cta_headn[blockIdx.x];   // reserved tiles, first visit only
     for (;;) {
@@ -89,7 +95,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
             int t0, t1;
             if (headn > 0) { t0 = head; t1 = head + headn; headn = 0; }
             else {
-                if (tid == 0) s_g = atomicAdd(&L.next[u], chunk);
+                if (tid == 0) s_g = atomicAdd(&nxt[u], chunk);
                 __syncthreads();
                 t0 = s_g;
                 __syncthreads();
@@ -135,7 +141,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
         }
         if (mine > 0) {
             // merge the four warps, write the visit's partial into a fresh slot of the unit
-            if (tid == 0) s_g = atomicAdd(&L.cnt[u].y, 1);
+            if (tid == 0) s_g = atomicAdd(&cnt[u].y, 1);
             if (lane == 0) {
 #pragma unroll
                 for (int h = 0; h < G; ++h) { xm[warp][h] = m[h]; xl[warp][h] = l[h]; }
@@ -168,14 +174,14 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
             __threadfence();
             __syncthreads();
             // the delivery that completes the unit's tile count runs its tail
-            if (tid == 0) s_last = (atomicAdd(&L.cnt[u].x, mine) + mine == total);
+            if (tid == 0) s_last = (atomicAdd(&cnt[u].x, mine) + mine == total);
             __syncthreads();
             if (s_last && !p.defer_tails) {
                 __threadfence();
                 constexpr int GB = G <= 4 ? 4 : 8;
                 TailPre<kSimtThreads, GB> pre;
                 tail_prefetch<T, kSimtThreads, GB>(p, u, tsm, tid, pre);
-                unit_tail<T, kSimtThreads, 1, GB>(p, u, __ldcg(&L.cnt[u].y), pre, tsm, tid);
+                unit_tail<T, kSimtThreads, 1, GB>(p, u, __ldcg(&cnt[u].y), pre, tsm, tid);
             }
             __syncthreads();
         }
@@ -185,7 +191,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
             for (int k = 1; k < U; ++k) {
                 const int cand = (u + k) % U;
                 const int nd = min(L.n_dec[cand], p.cap - (dec ? 1 : 0));
-                if (__ldcg(&L.next[cand]) < unit_tiles(L.unit_lp[cand], nd)) { found = cand; break; }
+                if (__ldcg(&nxt[cand]) < unit_tiles(L.unit_lp[cand], nd)) { found = cand; break; }
             }
             s_u = found;
         }

@@ -40,6 +40,7 @@ struct TailSmem {
     int hist[256];
     int cnt[3][NT / 32];
     int misc[4];
+    int par;                 // parity of this launch: which copy of the unit counters is in use
 };
 
 __device__ inline void copy_row_swizzled(uint8_t* pool, size_t unit_base, int rowb, int src, int dst,
@@ -82,9 +83,10 @@ __device__ inline void load_elems(const T* ptr, float (&f)[N]) {
 }
 
 // The unit is complete: prepare the idle copy of its counters for the next launch.
-__device__ inline void rewind_unit(const LayerDev& L, int u) {
-    L.next_idle[u] = L.unit_next0[u];
-    L.cnt_idle[u] = make_int2(0, 0);
+__device__ inline void rewind_unit(const LayerDev& L, int u, int par) {
+    const int idle = (par ^ 1) * L.n_units + u;
+    L.next[idle] = L.unit_next0[u];
+    L.cnt[idle] = make_int2(0, 0);
 }
 
 // What a tail can fetch before its unit is complete (nothing here is written by the step
@@ -310,7 +312,7 @@ __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB
     if (!dec) {
         finish_out();
         if (tid == 0) MKV_TR(11);
-        if (tid == 0) rewind_unit(L, u);
+        if (tid == 0) rewind_unit(L, u, sm.par);
         return;
     }
     if (tid == 0) MKV_TR(11);
@@ -393,7 +395,7 @@ __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB
         if (warp == (NW > 1 ? 1 : 0)) store_row_swizzled(L.Vd, ubase, rowb, vnew, n_old, lane);
         if (tid == NT - 1) { score[n_old] = ab_new; pos[n_old] = t; keys[n_old] = key_new; }
         if (k == 0) {
-            if (tid == 0) rewind_unit(L, u);
+            if (tid == 0) rewind_unit(L, u, sm.par);
             return;
         }
     }
@@ -424,7 +426,7 @@ __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB
             if (warp == (NW > 1 ? 1 : 0)) store_row_swizzled(L.Vd, ubase, rowb, vnew, e, lane);
             if (tid == NT - 1) { score[e] = ab_new; pos[e] = t; }
         }
-        if (tid == 0) rewind_unit(L, u);
+        if (tid == 0) rewind_unit(L, u, sm.par);
         return;
     }
 
@@ -500,7 +502,7 @@ __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB
             if (lane == 0) { score[dst] = score[src]; pos[dst] = pos[src]; }
         }
     }
-    if (tid == 0) rewind_unit(L, u);
+    if (tid == 0) rewind_unit(L, u, sm.par);
 }
 
 }  // namespace mkv

@@ -370,3 +370,64 @@ def test_per_head_prefill_lengths_like_a_compressed_prompt():
     ctx.status_sync()
     ctx.close()
     assert worst_out <= 2e-3 and worst_sc <= 1e-4, (worst_out, worst_sc)
+
+
+@pytest.mark.parametrize("case", ["mma_group", "simt_f32", "mma_layer"])
+def test_recorded_steps_replay_as_a_cuda_graph(case):
+    """A recorded sequence of decode steps (an odd number, so consecutive replays start on
+    alternating copies of the work-sharing counters) replays as a CUDA graph: outputs of every
+    step and the pool after every replay against the oracle run step by step (Algorithm 1)."""
+    import torch
+    from oracle import mkv_oracle as O
+    mode, omode = mkv.MKV_SCORE_GROUP_MEAN, O.GROUP_MEAN
+    if case == "simt_f32":
+        w = CONFIGS["tiny"].with_(q_heads=6, kv_heads=2, batch=2, prefill=70, steps=64, budget=24, variant="hot")
+    else:
+        w = CONFIGS["llama_b1"].with_(batch=3, prefill=(100, 400), steps=64, budget=40, variant="hot", n_heavy=3)
+        if case == "mma_layer":
+            mode, omode = mkv.MKV_SCORE_LAYER_MEAN, O.LAYER_MEAN
+    ctx = make_context(w, score_mode=mode)
+    stream = BatchStream(w, 0)
+    oracles, _ = prefill_both(ctx, w, stream, mode=omode)
+    rep = lockstep(ctx, w, stream, oracles, 35)          # eager steps first: the pool is nearly full
+    assert rep.ok(), rep.failures[:5]
+    dt, dev, n_rec = ctx.torch_kv_dtype(), ctx.device, 3
+    B = len(oracles)
+    q_s = torch.zeros((n_rec, B, w.q_heads, w.head_dim), dtype=dt, device=dev)
+    k_s = torch.zeros((n_rec, B, w.kv_heads, w.head_dim), dtype=dt, device=dev)
+    v_s = torch.zeros_like(k_s)
+    out_s = torch.zeros((n_rec, B, w.q_heads, w.head_dim), dtype=torch.float32, device=dev)
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    recorded = False
+    tol = 1e-5 if w.dtype == "f32" else 2e-3
+    for replay in range(5):
+        qs, ks, vs = stream.next(n_rec)
+        q_s.copy_(torch.from_numpy(np.ascontiguousarray(qs, dtype=np.float32)).to(dev, dt))
+        k_s.copy_(torch.from_numpy(np.ascontiguousarray(ks, dtype=np.float32)).to(dev, dt))
+        v_s.copy_(torch.from_numpy(np.ascontiguousarray(vs, dtype=np.float32)).to(dev, dt))
+        torch.cuda.synchronize()
+        if not recorded:                                  # recording runs nothing: replay it below
+            with torch.cuda.graph(graph, stream=side):
+                for i in range(n_rec):
+                    ctx.decode_step(0, q_s[i], k_s[i], v_s[i], out_s[i])
+            recorded = True
+        graph.replay()
+        torch.cuda.synchronize()
+        got = out_s.to(torch.float64).cpu().numpy()
+        for i in range(n_rec):
+            for b in range(B):
+                ref = oracles[b].attend_update(qs[i, b], ks[i, b], vs[i, b])
+                oracles[b].evict()
+                rowmax = np.abs(ref).max(axis=1)
+                assert (np.abs(got[i, b] - ref).max(axis=1) <= tol * rowmax).all(), (replay, i, b)
+        for b in range(B):
+            for g in range(w.kv_heads):
+                pos, sc = ctx.decode_state(0, b, g)
+                opos, osc, _ = oracles[b].decode_state(g)
+                order, oorder = np.argsort(pos), np.argsort(opos)
+                np.testing.assert_array_equal(pos[order], opos[oorder])
+                np.testing.assert_allclose(sc[order], osc[oorder], rtol=1e-4)
+    ctx.status_sync()
+    ctx.close()
