@@ -72,8 +72,7 @@ typedef enum {
     MKV_SCORE_GROUP_MEAN = 0, /* per KV head: mean over its G query heads; each KV head
                                  scores and evicts on its own                           */
     MKV_SCORE_LAYER_MEAN = 1  /* as printed: mean over all H heads, one score vector per
-                                 (layer, sequence), all KV heads evict the same tokens;
-                                 with more than one KV head a step is two kernels       */
+                                 (layer, sequence), all KV heads evict the same tokens  */
 } mkv_score_mode;
 
 /* Kernel family used for the attention pass. */

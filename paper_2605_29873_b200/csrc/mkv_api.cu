@@ -230,8 +230,8 @@ Params make_params(const mkv_ctx* c, int layer, const void* q, const void* k_new
     p.beta = c->beta;
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c->head_dim));
     p.mode = mode;
-    // Eq. 4 over all heads of the layer needs every KV head of a sequence: a second kernel
-    p.defer_tails = (mode == kModeDecode && c->score_mode == MKV_SCORE_LAYER_MEAN && c->kv_heads > 1) ? 1 : 0;
+    // Eq. 4 over all heads of the layer: the tails of a sequence's KV heads work together
+    p.layer_mean = (mode == kModeDecode && c->score_mode == MKV_SCORE_LAYER_MEAN && c->kv_heads > 1) ? 1 : 0;
     p.out_f32 = (c->out_dtype == MKV_F32);
     p.launch_parity = (int)(c->launches & 1);
     return p;
@@ -244,10 +244,6 @@ mkv_status launch_step(mkv_ctx* c, int layer, const Params& p, cudaStream_t st) 
     cudaError_t e = c->use_mma ? launch_mma(p, st, overlap) : launch_simt(p, c->kv_dtype, st);
     if (e != cudaSuccess) return MKV_ERR_CUDA;
     c->launches += 1;
-    if (p.defer_tails) {
-        if (launch_layer_tail(p, c->kv_dtype, st) != cudaSuccess) return MKV_ERR_CUDA;
-        c->launches += 1;
-    }
     c->stepped[layer] = 1;
     return MKV_OK;
 }
@@ -316,7 +312,6 @@ mkv_status mkv_create(int layers, int q_heads, int kv_heads, int head_dim, int b
     if (flags & ~MKV_FLAG_RECORD_PROBS) return MKV_ERR_INVALID_ARG;
     if (!workspace || device < 0) return MKV_ERR_INVALID_ARG;
     const int G = q_heads / kv_heads;
-    if (score_mode == MKV_SCORE_LAYER_MEAN && kv_heads != 1 && !layer_tail_supported(q_heads, G)) return MKV_ERR_UNSUPPORTED;
     const bool mma_ok = mma_supported(kv_dtype, head_dim, G);
     const bool simt_ok = simt_supported(kv_dtype, head_dim, G);
     bool use_mma;

@@ -102,7 +102,7 @@ struct Params {
     float scale_log2;  // log2(e) / sqrt(head_dim)
     int mode;
     int out_f32;
-    int defer_tails;   // the unit tails are left to a following kernel (layer-wide score mode)
+    int layer_mean;    // Eq. 4 over all heads of the layer: one score vector per sequence, shared eviction
     int launch_parity; // launches of the context so far, modulo 2 (diagnostic builds keep two trace sets)
 };
 

@@ -10,7 +10,5 @@ bool simt_supported(int kv_dtype, int head_dim, int group);
 cudaError_t launch_simt(const Params& p, int kv_dtype, cudaStream_t stream);
 bool mma_supported(int kv_dtype, int head_dim, int group);
 cudaError_t launch_mma(const Params& p, cudaStream_t stream, bool overlap);
-bool layer_tail_supported(int q_heads, int group);
-cudaError_t launch_layer_tail(const Params& p, int kv_dtype, cudaStream_t stream);
 cudaError_t mma_configure();   // one-time function attributes (dynamic shared memory)
 }  // namespace mkv

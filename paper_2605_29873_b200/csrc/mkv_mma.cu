@@ -38,6 +38,7 @@
 
 #include "mkv_launch.h"
 #include "mkv_ptx.cuh"
+#include "mkv_layer_tail.cuh"
 #include "mkv_tail.cuh"
 
 namespace mkv {
@@ -118,13 +119,14 @@ __device__ inline bool wait_or_abort(uint32_t bar, uint32_t parity, Control* ctl
 // streamed the group already fetches what its tail needs and the step does not change
 // (tail_prefetch); thread 0 then watches the unit's counters, which arrive as one 8-byte
 // word (tiles delivered, partial slots taken).
-template <int GB>
+// LAYER: the tails of a sequence's KV heads score together (Eq. 4 over all heads of the layer).
+template <int GB, bool LAYER>
 __device__ void tail_group(const Params& p, Control* ctl, TailSmem<kTailThreads>* tsm, int tt) {
     const LayerDev& L = p.L;
     const bool dec = (p.mode == kModeDecode);
     for (int u = blockIdx.x; u < L.n_units; u += gridDim.x) {
         TailPre<kTailThreads, GB> pre;
-        tail_prefetch<__nv_bfloat16, kTailThreads, GB>(p, u, *tsm, tt, pre);
+        tail_prefetch<__nv_bfloat16, kTailThreads, GB, LAYER>(p, u, *tsm, tt, pre);
         if (tt == 0) {
             const int total = unit_tiles(L.unit_lp[u], min(pre.n_dec, p.cap - (dec ? 1 : 0)));
             const unsigned long long t0 = ptx::globaltimer_ns();
@@ -152,11 +154,13 @@ __device__ void tail_group(const Params& p, Control* ctl, TailSmem<kTailThreads>
         if (slots < 0) break;
         __threadfence();
         if (tt == 0) MKV_TR_ADD(6, 1);
-        unit_tail<__nv_bfloat16, kTailThreads, 1, GB>(p, u, slots, pre, *tsm, tt);
+        if constexpr (LAYER) layer_unit_tail<__nv_bfloat16, kTailThreads, 1, GB>(p, u, slots, pre, *tsm, tt);
+        else unit_tail<__nv_bfloat16, kTailThreads, 1, GB>(p, u, slots, pre, *tsm, tt);
         if (tt == 0) MKV_TR(5);
     }
 }
 
+template <bool LAYER>
 __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const int nst) {
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t* const stages = smem;
@@ -608,10 +612,9 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         // tiles and runs the tail the moment the count is complete, so no CTA ever has two
         // tails due at once (as long as there are at least as many CTAs as units) and nothing
         // has to be announced or claimed.
-        if (p.defer_tails) return;     // a following kernel scores the whole layer at once
         ptx::griddep_wait();
-        if (G <= 4) tail_group<4>(p, ctl, tsm, tid - kTailTid0);
-        else tail_group<8>(p, ctl, tsm, tid - kTailTid0);
+        if (G <= 4) tail_group<4, LAYER>(p, ctl, tsm, tid - kTailTid0);
+        else tail_group<8, LAYER>(p, ctl, tsm, tid - kTailTid0);
     }
 }
 
@@ -631,7 +634,9 @@ bool mma_supported(int kv_dtype, int head_dim, int group) {
 
 cudaError_t mma_configure() {
     if (const char* e = std::getenv("MKV_STAGES")) g_stages = max(2, min(kMaxStages, atoi(e)));
-    return cudaFuncSetAttribute(mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(g_stages));
+    cudaError_t e = cudaFuncSetAttribute(mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(g_stages));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(g_stages));
 }
 
 // overlap: launch with programmatic stream serialization, i.e. this kernel's CTAs may start
@@ -649,7 +654,9 @@ cudaError_t launch_mma(const Params& p, cudaStream_t st, bool overlap) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = overlap ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, mma_kernel, p, g_stages);
+    // the layer-wide score mode has its own instantiation, so that neither carries the other's tail
+    if (p.layer_mean) return cudaLaunchKernelEx(&cfg, mma_kernel<true>, p, g_stages);
+    return cudaLaunchKernelEx(&cfg, mma_kernel<false>, p, g_stages);
 }
 
 }  // namespace mkv

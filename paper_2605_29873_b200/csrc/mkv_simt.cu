@@ -11,6 +11,7 @@
 // are merged in shared memory and the CTA writes one partial with its tile count; the
 // delivery that completes the unit runs its tail.
 #include "mkv_launch.h"
+#include "mkv_layer_tail.cuh"
 #include "mkv_tail.cuh"
 
 namespace mkv {
@@ -176,12 +177,17 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
             // the delivery that completes the unit's tile count runs its tail
             if (tid == 0) s_last = (atomicAdd(&cnt[u].x, mine) + mine == total);
             __syncthreads();
-            if (s_last && !p.defer_tails) {
+            if (s_last) {
                 __threadfence();
                 constexpr int GB = G <= 4 ? 4 : 8;
                 TailPre<kSimtThreads, GB> pre;
-                tail_prefetch<T, kSimtThreads, GB>(p, u, tsm, tid, pre);
-                unit_tail<T, kSimtThreads, 1, GB>(p, u, __ldcg(&cnt[u].y), pre, tsm, tid);
+                if (p.layer_mean) {
+                    tail_prefetch<T, kSimtThreads, GB, true>(p, u, tsm, tid, pre);
+                    layer_unit_tail<T, kSimtThreads, 1, GB>(p, u, __ldcg(&cnt[u].y), pre, tsm, tid);
+                } else {
+                    tail_prefetch<T, kSimtThreads, GB>(p, u, tsm, tid, pre);
+                    unit_tail<T, kSimtThreads, 1, GB>(p, u, __ldcg(&cnt[u].y), pre, tsm, tid);
+                }
             }
             __syncthreads();
         }

@@ -134,7 +134,8 @@ __device__ inline void load_vec(const int32_t* src, int (&dst)[TW]) {
 }
 
 // GB: compile-time bound of the group size G (4 or 8); it sizes the register staging.
-template <typename T, int NT, int GB>
+// LAYER: the scores are updated later, for all KV heads of the sequence at once; none fetched here.
+template <typename T, int NT, int GB, bool LAYER = false>
 __device__ void tail_prefetch(const Params& p, int u, TailSmem<NT>& sm, int tid, TailPre<NT, GB>& pre) {
     constexpr int TW = TailPre<NT, GB>::TW, OCB = TailPre<NT, GB>::OCB, NW = NT / 32;
     const LayerDev& L = p.L;
@@ -151,10 +152,12 @@ __device__ void tail_prefetch(const Params& p, int u, TailSmem<NT>& sm, int tid,
     const float* score = L.score + (size_t)u * ls;
     const int32_t* pos = L.pos + (size_t)u * ls;
     const int n_old = min(pre.n_dec, p.cap - 1);
+    if constexpr (!LAYER) {
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
-        const int i0 = TW * (tid + k * NT);
-        if (i0 < n_old) { load_vec<TW>(score + i0, pre.sc[k]); load_vec<TW>(pos + i0, pre.ps[k]); }
+        for (int k = 0; k < 2; ++k) {
+            const int i0 = TW * (tid + k * NT);
+            if (i0 < n_old) { load_vec<TW>(score + i0, pre.sc[k]); load_vec<TW>(pos + i0, pre.ps[k]); }
+        }
     }
     const int ne = G * D / 4;
 #pragma unroll
@@ -183,7 +186,12 @@ __device__ void tail_prefetch(const Params& p, int u, TailSmem<NT>& sm, int tid,
 }
 
 // The tail proper; P = partial slots the unit's visits took.
-template <typename T, int NT, int BAR, int GB>
+// LAYER (score mode "mean over all heads of the layer"): the tail stops after `out` and the
+// probabilities.  Per decode token it leaves the SUM over the unit's G heads of the normalised
+// probabilities (the fresh token's at index n_old) in the first of the unit's logit rows, whose
+// entries the same thread has just consumed; scores, selection and compaction follow for all
+// KV heads of the sequence together (layer_finish).
+template <typename T, int NT, int BAR, int GB, bool LAYER = false>
 __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB>& pre, TailSmem<NT>& sm, int tid) {
     const LayerDev& L = p.L;
     const int G = p.group, D = p.head_dim, cap = p.cap, ls = p.lstride;
@@ -205,6 +213,7 @@ __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB
     float* score = L.score + (size_t)u * ls;
     int32_t* pos = L.pos + (size_t)u * ls;
     const float* lg = L.logit + ((size_t)b * p.q_heads + (size_t)g * G) * ls;
+    float* psum = L.logit + ((size_t)b * p.q_heads + (size_t)g * G) * ls;   // LAYER only
     const float* po_base = L.part_o + (size_t)part0 * G * D;
     const size_t pstride = (size_t)G * D;
     const int ne = G * D / 4;                           // float4 elements of one partial / of `out`
@@ -321,9 +330,9 @@ __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB
     const int k = max(0, n - p.budget);
     const float inv_g = 1.0f / (float)G;
     unsigned long long* keys = L.keys + (size_t)u * cap;
-    float ab_new = 0.f;
-    for (int h = 0; h < G; ++h) ab_new += sm.wnew[h] * sm.invL[h];
-    ab_new *= inv_g;                                  // Eq. 6: I_fresh = alpha * 0 + abar_fresh
+    float sum_new = 0.f;
+    for (int h = 0; h < G; ++h) sum_new = fmaf(sm.wnew[h], sm.invL[h], sum_new);
+    const float ab_new = sum_new * inv_g;             // Eq. 6: I_fresh = alpha * 0 + abar_fresh
     const unsigned long long key_new = ((unsigned long long)__float_as_uint(ab_new) << 32) | (unsigned)t;
     unsigned long long best_key = ~0ull;
     int best_slot = -1;
@@ -339,6 +348,12 @@ __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB
 #pragma unroll
                 for (int j = 0; j < TW; ++j) ab[j] = fmaf(fast_exp2(r.lgv[h][j] - Mh), iLh, ab[j]);
             }
+        }
+        if constexpr (LAYER) {
+            // whole vectors: the row is lstride (a multiple of 4) floats long, so the tail is in bounds
+            if constexpr (TW == 4) *reinterpret_cast<float4*>(psum + i0) = make_float4(ab[0], ab[1], ab[2], ab[3]);
+            else *reinterpret_cast<float2*>(psum + i0) = make_float2(ab[0], ab[1]);
+            return;
         }
 #pragma unroll
         for (int j = 0; j < TW; ++j) {
@@ -373,7 +388,7 @@ __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB
         if (pass == 1) {
 #pragma unroll
             for (int j = 0; j < TW; ++j) { sc[j] = pre.sc[1][j]; ps[j] = pre.ps[1][j]; }
-        } else if (i0 < n_old) {
+        } else if (!LAYER && i0 < n_old) {
             load_vec<TW>(score + i0, sc);
             load_vec<TW>(pos + i0, ps);
         }
@@ -382,6 +397,11 @@ __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB
     }
     if (!out_done) finish_out();
     if (tid == 0) MKV_TR(12);
+    if constexpr (LAYER) {
+        bar_sync(BAR, NT);                            // every vector store above is done ...
+        if (tid == NT - 1) psum[n_old] = sum_new;     // ... before the fresh token's sum lands
+        return;
+    }
     if (tid == NT - 1) {                              // the fresh token sits (virtually) in slot n_old
         if (key_new < best_key) { best_key = key_new; best_slot = n_old; }
         if (L.abar) L.abar[(size_t)u * cap + n_old] = ab_new;
