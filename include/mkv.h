@@ -155,7 +155,7 @@ mkv_status mkv_prefill(mkv_ctx* ctx, int layer, const void* K, const void* V,
 
 /*
  * The same with one prompt length per (sequence, KV head) unit: the shape of a frozen pool
- * that a per-head prefill compressor (SnapKV- or PyramidKV-like; Sec. 5.4 of the paper runs
+ * that a per-head prefill compressor (SnapKV- or PyramidKV-like; Sec. 6.3 of the paper runs
  * Moment-KV on top of such pools) has already thinned out.  The compressors themselves are
  * not part of this library: K and V hold, for unit (b, g), its retained rows first.
  *   unit_lens     host pointer, [batch * kv_heads]; unit (b, g) uses rows [0, unit_lens[b*kv_heads+g])

@@ -312,7 +312,7 @@ def test_head_averaged_probabilities_match_eq4(mode):
 def test_per_head_prefill_lengths_like_a_compressed_prompt():
     """mkv_prefill_units: every (sequence, KV head) unit keeps its own number of prompt rows and
     the two layers differ as well -- the shape of a prefill pool that a per-head / per-layer
-    compressor has thinned out (the paper's plug-in setting, Sec. 5.4).  In the group score mode
+    compressor has thinned out (the paper's plug-in setting, Sec. 6.3).  In the group score mode
     each unit is an independent instance of Algorithm 1, so the oracle is one single-KV-head
     instance per unit."""
     import torch
