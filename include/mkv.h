@@ -84,7 +84,8 @@ typedef enum {
 
 /* flags for mkv_create */
 #define MKV_FLAG_RECORD_PROBS 1u /* keep the head-averaged decode probabilities of the last
-                                    step (Eq. 4) for mkv_get_last_probs()               */
+                                    step (Eq. 4) and their position ids, for
+                                    mkv_get_last_probs() and mkv_recency_diagnostics()  */
 
 /*
  * Size in bytes of the workspace mkv_create() needs for these parameters
@@ -242,6 +243,30 @@ mkv_status mkv_attend_noalloc(const void* q, const void* K, const void* V, void*
 /* Number of kernels this context has launched so far (host counter). */
 int64_t mkv_launch_count(const mkv_ctx* ctx);
 
+/*
+ * Recency-window attention diagnostics of the last decode step of `layer` (the analysis of
+ * Sec. 3.2 and Sec. 7.1 of the paper: how a step's attention is spread over the most recently
+ * decoded tokens), from the probabilities the step recorded (MKV_FLAG_RECORD_PROBS, else
+ * MKV_ERR_BAD_STATE).  The paper shows figures, no formulas; the quantities are defined here.
+ * For every (sequence, KV head) unit u = b * kv_heads + kv_head, with t the id of the last step
+ * and the window = the cached decode tokens (before that step's eviction) whose position id
+ * lies in (t - window, t]:
+ *   count[u]          number of tokens in the window (<= window)
+ *   mass[u]           attention they received together, head-averaged as in Eq. 4 (a share
+ *                     of 1; the rest went to older decode tokens and to the prompt)
+ *   curve[u][j]       share of mass[u] held by the j+1 most attended tokens of the window,
+ *                     j < count[u]; entries from count[u] to window-1 are set to 0.  Uniform
+ *                     attention would give (j+1)/count[u].
+ * In the score mode MKV_SCORE_LAYER_MEAN the values are those of the whole layer, equal in
+ * every KV head of a sequence.  Before the first step all outputs are 0.
+ * mass: device float [batch*kv_heads]; count: device int32 [batch*kv_heads]; curve: device
+ * float [batch*kv_heads][window]; all owned by the caller, written by a kernel on `stream`
+ * (asynchronous, allocation-free).  window >= 1; min(window, budget + 1) <= 8192, else
+ * MKV_ERR_UNSUPPORTED.  Not part of the decode step: nothing is computed unless called.
+ */
+mkv_status mkv_recency_diagnostics(mkv_ctx* ctx, int layer, int window, float* mass, int32_t* count,
+                                   float* curve, void* stream);
+
 /* ---- inspection: synchronous (device-wide sync + D2H), for tests and debugging ---- */
 
 /* Decode pool of (layer, b, kv_head): *n tokens; pos/score (host, `cap` entries) may be
@@ -251,10 +276,11 @@ mkv_status mkv_get_decode_state(mkv_ctx* ctx, int layer, int b, int kv_head, int
 /* Tokens the last step evicted from that pool, with their scores at eviction. */
 mkv_status mkv_get_last_evicted(mkv_ctx* ctx, int layer, int b, int kv_head, int32_t* k,
                                 int32_t* pos, float* score, int cap);
-/* Eq. 4 values of the last step per slot, pre-eviction order (needs MKV_FLAG_RECORD_PROBS);
+/* Eq. 4 values of the last step per slot, pre-eviction order, and the position ids of those
+ * slots (needs MKV_FLAG_RECORD_PROBS; abar, pos: host, `cap` entries, either may be NULL);
  * *n receives the pre-eviction token count. */
 mkv_status mkv_get_last_probs(mkv_ctx* ctx, int layer, int b, int kv_head, int32_t* n,
-                              float* abar, int cap);
+                              float* abar, int32_t* pos, int cap);
 /* Copy a pool's rows out in plain [token][head_dim] layout (kv_dtype).  pool 0 = prefill,
  * 1 = decode.  *n receives the token count; at most cap_tokens rows are written. */
 mkv_status mkv_read_kv(mkv_ctx* ctx, int layer, int b, int kv_head, int pool, int32_t* n,

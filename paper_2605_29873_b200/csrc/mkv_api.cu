@@ -22,7 +22,7 @@ inline int round4(int a) { return (a + 3) / 4 * 4; }
 inline int elem_size(int dt) { return dt == MKV_BF16 ? 2 : 4; }
 
 struct LayerOff {
-    size_t Kp, Vp, Kd, Vd, score, pos, n_dec, abar, n_prev, ev_k, ev_pos, ev_score, cta_unit0, cta_head0,
+    size_t Kp, Vp, Kd, Vd, score, pos, n_dec, abar, abar_pos, n_prev, ev_k, ev_pos, ev_score, cta_unit0, cta_head0,
         cta_headn, unit_lp, unit_next0, next, cnt, launch_no, unit_step, seq_ticket, end;
 };
 // Scratch that lives for one step only, shared by all layers of the context (calls on a
@@ -78,6 +78,7 @@ bool make_layout(int layers, int batch, int q_heads, int kv_heads, int head_dim,
     L.lo.pos = take(U * L.lstride * 4);
     L.lo.n_dec = take(U * 4);
     L.lo.abar = take(U * C * 4);
+    L.lo.abar_pos = take(U * C * 4);
     L.lo.n_prev = take(U * 4);
     L.lo.ev_k = take(U * 4);
     L.lo.ev_pos = take(U * C * 4);
@@ -193,6 +194,7 @@ LayerDev layer_dev(const mkv_ctx* c, int layer) {
     d.n_dec = (int32_t*)(base + o.n_dec);
     d.logit = (float*)(sb + so.logit);
     d.abar = (c->flags & MKV_FLAG_RECORD_PROBS) ? (float*)(base + o.abar) : nullptr;
+    d.abar_pos = (int32_t*)(base + o.abar_pos);
     d.n_prev = (int32_t*)(base + o.n_prev);
     d.ev_k = (int32_t*)(base + o.ev_k);
     d.ev_pos = (int32_t*)(base + o.ev_pos);
@@ -540,7 +542,7 @@ mkv_status mkv_get_last_evicted(mkv_ctx* c, int layer, int b, int g, int32_t* k,
     return MKV_OK;
 }
 
-mkv_status mkv_get_last_probs(mkv_ctx* c, int layer, int b, int g, int32_t* n, float* abar, int cap) {
+mkv_status mkv_get_last_probs(mkv_ctx* c, int layer, int b, int g, int32_t* n, float* abar, int32_t* pos, int cap) {
     mkv_status s = unit_args(c, layer, b, g);
     if (s != MKV_OK) return s;
     if (!n) return MKV_ERR_INVALID_ARG;
@@ -550,8 +552,22 @@ mkv_status mkv_get_last_probs(mkv_ctx* c, int layer, int b, int g, int32_t* n, f
     const LayerDev d = layer_dev(c, layer);
     const int u = b * c->kv_heads + g;
     MKV_D2H(n, d.n_prev + u, 4);
-    if (abar && *n > cap) return MKV_ERR_CAPACITY;
+    if ((abar || pos) && *n > cap) return MKV_ERR_CAPACITY;
     if (abar) MKV_D2H(abar, d.abar + (size_t)u * c->lay.cap, (size_t)*n * 4);
+    if (pos) MKV_D2H(pos, d.abar_pos + (size_t)u * c->lay.cap, (size_t)*n * 4);
+    return MKV_OK;
+}
+
+mkv_status mkv_recency_diagnostics(mkv_ctx* c, int layer, int window, float* mass, int32_t* count, float* curve,
+                                   void* stream) {
+    if (!layer_ok(c, layer) || window < 1 || !mass || !count || !curve) return MKV_ERR_INVALID_ARG;
+    if (!c->prefilled[layer] || !(c->flags & MKV_FLAG_RECORD_PROBS)) return MKV_ERR_BAD_STATE;
+    if (std::min(window, c->lay.cap) > diag_max_tokens()) return MKV_ERR_UNSUPPORTED;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MKV_ERR_CUDA;
+    if (launch_diag(layer_dev(c, layer), c->lay.cap, window, mass, count, curve, (cudaStream_t)stream) != cudaSuccess)
+        return MKV_ERR_CUDA;
+    c->launches += 1;
     return MKV_OK;
 }
 

@@ -59,7 +59,8 @@ struct LayerDev {
     int32_t* pos;
     int32_t* n_dec;
     float* logit;      // [batch*q_heads][lstride] raw logits (log2 units) of decode-pool tokens
-    float* abar;       // [units][cap] or nullptr
+    float* abar;       // [units][cap] or nullptr: Eq. 4 values of the last step, slot order before its eviction
+    int32_t* abar_pos; // [units][cap], with abar: the position ids of those slots
     int32_t* n_prev;   // [units] decode count (fresh token included) before the last eviction
     int32_t* ev_k;     // [units] tokens evicted by the last step
     int32_t* ev_pos;   // [units][cap]

@@ -10,5 +10,9 @@ bool simt_supported(int kv_dtype, int head_dim, int group);
 cudaError_t launch_simt(const Params& p, int kv_dtype, cudaStream_t stream);
 bool mma_supported(int kv_dtype, int head_dim, int group);
 cudaError_t launch_mma(const Params& p, cudaStream_t stream, bool overlap);
+// recency-window diagnostics over the recorded probabilities of the last step
+int diag_max_tokens();
+cudaError_t launch_diag(const LayerDev& L, int cap, int window, float* mass, int32_t* count, float* curve,
+                        cudaStream_t stream);
 cudaError_t mma_configure();   // one-time function attributes (dynamic shared memory)
 }  // namespace mkv

@@ -102,7 +102,11 @@ __device__ void layer_finish(const Params& p, int u, const TailPre<NT, GB>& pre,
                 for (int j = 0; j < TW; ++j) if (i0 + j < n_old) sg[j] = nw[j];
             }
             if (L.abar)
-                for (int j = 0; j < TW; ++j) if (i0 + j < n_old) L.abar[(size_t)(u0 + g2) * cap + i0 + j] = ab[j];
+                for (int j = 0; j < TW; ++j)
+                    if (i0 + j < n_old) {
+                        L.abar[(size_t)(u0 + g2) * cap + i0 + j] = ab[j];
+                        L.abar_pos[(size_t)(u0 + g2) * cap + i0 + j] = ps[j];
+                    }
         }
 #pragma unroll
         for (int j = 0; j < TW; ++j) {
@@ -122,7 +126,10 @@ __device__ void layer_finish(const Params& p, int u, const TailPre<NT, GB>& pre,
     if (tid == NT - 1) {                               // the fresh token sits (virtually) in slot n_old
         if (key_new < best_key) { best_key = key_new; best_slot = n_old; }
         if (L.abar)
-            for (int g2 = 0; g2 < Hkv; ++g2) L.abar[(size_t)(u0 + g2) * cap + n_old] = ab_new;
+            for (int g2 = 0; g2 < Hkv; ++g2) {
+                L.abar[(size_t)(u0 + g2) * cap + n_old] = ab_new;
+                L.abar_pos[(size_t)(u0 + g2) * cap + n_old] = t;
+            }
     }
     for (int g2 = tid; g2 < Hkv; g2 += NT) {
         const int u2 = u0 + g2;

@@ -370,7 +370,7 @@ __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB
 #pragma unroll
         for (int j = 0; j < TW; ++j) {
             if (i0 + j < n_old) {
-                if (L.abar) L.abar[(size_t)u * cap + i0 + j] = ab[j];
+                if (L.abar) { L.abar[(size_t)u * cap + i0 + j] = ab[j]; L.abar_pos[(size_t)u * cap + i0 + j] = ps[j]; }
                 const unsigned long long key = ((unsigned long long)__float_as_uint(nw[j]) << 32) | (unsigned)ps[j];
                 if (k > 1) keys[i0 + j] = key;
                 if (key < best_key) { best_key = key; best_slot = i0 + j; }
@@ -404,7 +404,7 @@ __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB
     }
     if (tid == NT - 1) {                              // the fresh token sits (virtually) in slot n_old
         if (key_new < best_key) { best_key = key_new; best_slot = n_old; }
-        if (L.abar) L.abar[(size_t)u * cap + n_old] = ab_new;
+        if (L.abar) { L.abar[(size_t)u * cap + n_old] = ab_new; L.abar_pos[(size_t)u * cap + n_old] = t; }
     }
     if (tid == 0) { L.n_prev[u] = n; L.ev_k[u] = k; L.n_dec[u] = n - k; L.unit_step[u] = t + 1; }
 

@@ -22,6 +22,7 @@ EXPORTED_SYMBOLS = [
     "mkv_decode_step", "mkv_decode_step_host", "mkv_attend_only", "mkv_set_budget", "mkv_reset",
     "mkv_status_sync", "mkv_launch_count", "mkv_get_decode_state", "mkv_get_last_evicted",
     "mkv_get_last_probs", "mkv_read_kv", "mkv_get_step", "mkv_status_string", "mkv_attend_noalloc", "mkv_plan_starts", "mkv_prefill_units",
+    "mkv_recency_diagnostics",
 ]
 
 
@@ -64,7 +65,8 @@ def load_library(path: str | None = None):
     L.mkv_launch_count.argtypes = [vp]
     L.mkv_get_decode_state.argtypes = [vp, C.c_int, C.c_int, C.c_int, i32p, i32p, f32p, C.c_int]
     L.mkv_get_last_evicted.argtypes = [vp, C.c_int, C.c_int, C.c_int, i32p, i32p, f32p, C.c_int]
-    L.mkv_get_last_probs.argtypes = [vp, C.c_int, C.c_int, C.c_int, i32p, f32p, C.c_int]
+    L.mkv_get_last_probs.argtypes = [vp, C.c_int, C.c_int, C.c_int, i32p, f32p, i32p, C.c_int]
+    L.mkv_recency_diagnostics.argtypes = [vp, C.c_int, C.c_int, vp, vp, vp, vp]
     L.mkv_read_kv.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, i32p, vp, vp, C.c_int]
     L.mkv_get_step.argtypes = [vp, C.c_int, C.POINTER(C.c_int64)]
     L.mkv_attend_noalloc.argtypes = [vp, vp, vp, vp] + [C.c_int] * 9 + [vp]
@@ -253,13 +255,21 @@ class MomentKV:
                                             sc.ctypes.data_as(C.POINTER(C.c_float)), cap), "mkv_get_last_evicted")
         return pos[: k.value].copy(), sc[: k.value].copy()
 
-    def last_probs(self, layer, b, g):
+    def last_probs(self, layer, b, g, with_pos=False):
         cap = self.budget_cap()
         n = C.c_int32(0)
         ab = np.zeros(cap, dtype=np.float32)
+        pos = np.zeros(cap, dtype=np.int32)
         _check(self._L.mkv_get_last_probs(self._ctx, layer, b, g, C.byref(n), ab.ctypes.data_as(C.POINTER(C.c_float)),
-                                          cap), "mkv_get_last_probs")
+                                          pos.ctypes.data_as(C.POINTER(C.c_int32)), cap), "mkv_get_last_probs")
+        if with_pos:
+            return ab[: n.value].copy(), pos[: n.value].copy()
         return ab[: n.value].copy()
+
+    def recency_diagnostics(self, layer, window, mass, count, curve, stream=None):
+        """mass: float32 [units], count: int32 [units], curve: float32 [units, window] device tensors."""
+        _check(self._L.mkv_recency_diagnostics(self._ctx, layer, int(window), _ptr(mass), _ptr(count), _ptr(curve),
+                                               self._stream(stream)), "mkv_recency_diagnostics")
 
     def read_kv(self, layer, b, g, pool):
         """Rows of a pool as float64 numpy arrays [n, head_dim] (exact: widening only)."""

@@ -431,3 +431,67 @@ def test_recorded_steps_replay_as_a_cuda_graph(case):
                 np.testing.assert_allclose(sc[order], osc[oorder], rtol=1e-4)
     ctx.status_sync()
     ctx.close()
+
+
+@pytest.mark.parametrize("mode", ["group", "layer"])
+def test_recency_window_diagnostics(mode):
+    """mkv_recency_diagnostics (Sec. 3.2 / Sec. 7.1 analysis) against the oracle: the attention
+    mass of the last W decoded tokens, their number, and the cumulative share of the most attended
+    ones.  Two comparisons per step: the oracle fed the GPU's own recorded probabilities and
+    position ids (sorting, windowing and summation: 1e-6), and the oracle fed its own fp64
+    probabilities (the whole chain: the tolerance of the recorded probabilities, 3e-4)."""
+    import torch
+    from oracle import mkv_diagnostics as D
+    from oracle import mkv_oracle as O
+    w = CONFIGS["llama_b1"].with_(batch=2, prefill=(60, 150), steps=100, budget=70, variant="hot", n_heavy=2)
+    smode = mkv.MKV_SCORE_LAYER_MEAN if mode == "layer" else mkv.MKV_SCORE_GROUP_MEAN
+    ctx = make_context(w, record_probs=True, score_mode=smode)
+    stream = BatchStream(w, 0)
+    oracles, _ = prefill_both(ctx, w, stream, mode=O.LAYER_MEAN if mode == "layer" else O.GROUP_MEAN)
+    dt, dev = ctx.torch_kv_dtype(), ctx.device
+    B, U = w.batch, w.batch * w.kv_heads
+    out = torch.zeros((B, w.q_heads, w.head_dim), dtype=torch.float32, device=dev)
+    qs, ks, vs = stream.next(w.steps)
+    windows = [1, 16, 256]                               # one token; inside the pool; wider than the pool
+    bufs = {W: (torch.full((U,), -1.0, device=dev), torch.full((U,), -1, dtype=torch.int32, device=dev),
+                torch.full((U, W), -1.0, device=dev)) for W in windows}
+    # before the first step everything is zero
+    ctx.recency_diagnostics(0, 16, *bufs[16])
+    torch.cuda.synchronize()
+    assert not bufs[16][0].any() and not bufs[16][1].any() and not bufs[16][2].any()
+    checked = 0
+    for i in range(w.steps):
+        ctx.decode_step(0, *(torch.from_numpy(np.ascontiguousarray(a[i], dtype=np.float32)).to(dev, dt)
+                             for a in (qs, ks, vs)), out)
+        for b in range(B):
+            oracles[b].attend_update(qs[i, b], ks[i, b], vs[i, b])
+        if i % 7 == 0 or i >= w.steps - 3:
+            for W in windows:
+                ctx.recency_diagnostics(0, W, *bufs[W])
+            torch.cuda.synchronize()
+            for W in windows:
+                mass, count, curve = (x.cpu().numpy() for x in bufs[W])
+                for b in range(B):
+                    for g in range(w.kv_heads):
+                        u = b * w.kv_heads + g
+                        g_ab, g_pos = ctx.last_probs(0, b, g, with_pos=True)
+                        m1, c1, cv1 = D.recency_window(g_ab, g_pos, i, W)          # GPU's own inputs
+                        o_pos, _, o_ab = oracles[b].decode_state(g)
+                        m2, c2, cv2 = D.recency_window(o_ab, o_pos, i, W)          # the oracle's
+                        assert count[u] == c1 == c2 <= min(W, len(o_pos))
+                        assert mass[u] == pytest.approx(m1, rel=1e-6) and mass[u] == pytest.approx(m2, rel=3e-4)
+                        np.testing.assert_allclose(curve[u, :c1], cv1, rtol=1e-6, atol=1e-7)
+                        np.testing.assert_allclose(curve[u, :c1], cv2, rtol=3e-4, atol=1e-6)
+                        assert not curve[u, c1:].any()
+                        checked += 1
+        for b in range(B):   # keep the oracle in step with the GPU's eviction choice
+            oracles[b].evict(force=[ctx.last_evicted(0, b, g)[0].astype(np.int64) for g in range(w.kv_heads)])
+    # argument and state errors
+    with pytest.raises(mkv.MkvError):
+        ctx.recency_diagnostics(0, 0, *bufs[16])
+    ctx.close()
+    plain = make_context(w)                              # probabilities not recorded
+    with pytest.raises(mkv.MkvError):
+        plain.recency_diagnostics(0, 16, *bufs[16])
+    plain.close()
+    assert checked > 100
