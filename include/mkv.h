@@ -101,7 +101,10 @@ size_t mkv_workspace_bytes(int layers, int batch, int q_heads, int kv_heads, int
  * inspection and tests).  The rows of a (sequence, KV head) unit form 64-row tiles, prefill
  * tiles first; CTAs are spread over the units in proportion to the units' tile counts and
  * each owns up to 3 reserved prefill tiles where it starts, the rest being handed out by
- * per-unit counters at run time.
+ * per-unit counters at run time, unit_chunk tiles per pull.  At most 32 CTAs start in one
+ * unit (the grid shrinks when few, long units would draw more), and a unit's chunk is sized so
+ * that the CTAs starting there plus the pulls of its counter stay within the 64 partial results
+ * a unit has room for.
  *   prefill_lens    host, [batch]
  *   n_ctas_max      upper bound of the grid (1..2048)
  *   n_ctas          host out: CTAs used
@@ -109,10 +112,11 @@ size_t mkv_workspace_bytes(int layers, int batch, int q_heads, int kv_heads, int
  *                   tile there, and how many tiles it has reserved (0 or 3)
  *   unit_next0      host out, [batch*kv_heads]: reserved tiles per unit = start value of the
  *                   unit's counter
+ *   unit_chunk      host out, [batch*kv_heads]: tiles per pull of the unit's counter (>= 2)
  */
 mkv_status mkv_plan_starts(int batch, int kv_heads, int budget, const int32_t* prefill_lens, int n_ctas_max,
                            int32_t* n_ctas, int32_t* cta_unit0, int32_t* cta_head0, int32_t* cta_headn,
-                           int32_t* unit_next0);
+                           int32_t* unit_next0, int32_t* unit_chunk);
 
 /* K+V bytes one cached token occupies over all layers (the paper's 128 KB/token). */
 size_t mkv_kv_bytes_per_token(int layers, int kv_heads, int head_dim, int kv_dtype);

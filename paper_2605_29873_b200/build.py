@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmkv.so")
 SOURCES = ["mkv_api.cu", "mkv_simt.cu", "mkv_mma.cu", "mkv_diag.cu", "mkv_noalloc.cu"]
-HEADERS = ["mkv_common.cuh", "mkv_tail.cuh", "mkv_ptx.cuh", "mkv_launch.h", os.path.join("..", "..", "include", "mkv.h")]
+HEADERS = ["mkv_common.cuh", "mkv_tail.cuh", "mkv_layer_tail.cuh", "mkv_ptx.cuh", "mkv_launch.h", os.path.join("..", "..", "include", "mkv.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",

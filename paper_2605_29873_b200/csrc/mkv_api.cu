@@ -23,7 +23,7 @@ inline int elem_size(int dt) { return dt == MKV_BF16 ? 2 : 4; }
 
 struct LayerOff {
     size_t Kp, Vp, Kd, Vd, score, pos, n_dec, abar, abar_pos, n_prev, ev_k, ev_pos, ev_score, cta_unit0, cta_head0,
-        cta_headn, unit_lp, unit_next0, next, cnt, launch_no, unit_step, seq_ticket, end;
+        cta_headn, unit_lp, unit_next0, unit_chunk, next, cnt, launch_no, unit_step, seq_ticket, end;
 };
 // Scratch that lives for one step only, shared by all layers of the context (calls on a
 // context are ordered on one stream, and a step touches it only after every earlier kernel
@@ -88,6 +88,7 @@ bool make_layout(int layers, int batch, int q_heads, int kv_heads, int head_dim,
     L.lo.cta_headn = take((size_t)kMaxCtas * 4);
     L.lo.unit_lp = take(U * 4);
     L.lo.unit_next0 = take(U * 4);
+    L.lo.unit_chunk = take(U * 4);
     L.lo.next = take(2 * U * 4);      // two copies each, alternating from launch to launch
     L.lo.cnt = take(2 * U * 8);
     L.lo.launch_no = take((size_t)kMaxCtas * 4);   // per CTA: launches since the prefill
@@ -127,9 +128,16 @@ __global__ void prefill_copy_kernel(const uint8_t* __restrict__ srcK, const uint
 // unit has that many prefill tiles left to give (these can be fetched before the previous
 // step has finished); everything else is handed out by the unit's counter, which
 // therefore starts behind the reserved tiles.  Returns the number of CTAs (the grid).
+//
+// Every visit of a unit by a CTA that covers at least one tile delivers one partial, and a unit
+// has room for kMaxParts of them.  Visits are bounded by the CTAs that start in the unit plus
+// the successful pulls of its counter, so the table keeps the first below kMaxHome (the grid
+// shrinks when few, long units would draw more) and sizes the unit's chunk -- tiles per pull --
+// so that the second stays below kMaxParts - 8 - (CTAs starting there).
 int build_start_table(int units, int budget, const int32_t* unit_lens, int n_ctas_max,
-                      std::vector<int32_t>& lp, std::vector<int32_t>& next0, std::vector<int32_t>& cta_unit0,
-                      std::vector<int32_t>& cta_head0, std::vector<int32_t>& cta_headn) {
+                      std::vector<int32_t>& lp, std::vector<int32_t>& next0, std::vector<int32_t>& chunk,
+                      std::vector<int32_t>& cta_unit0, std::vector<int32_t>& cta_head0,
+                      std::vector<int32_t>& cta_headn) {
     const int U = units;
     const int td = ceil_div(budget, kTileRows);
     lp.assign(U, 0);
@@ -140,7 +148,11 @@ int build_start_table(int units, int budget, const int32_t* unit_lens, int n_cta
         tile_begin[u + 1] = tile_begin[u] + ceil_div(lp[u], kTileRows) + td;
     }
     const long long t_all = tile_begin[U];
-    const int n_ctas = (int)std::max<long long>(1, std::min<long long>(n_ctas_max, t_all / 2));
+    long long t_max = 1;
+    for (int u = 0; u < U; ++u) t_max = std::max(t_max, tile_begin[u + 1] - tile_begin[u]);
+    // a unit of t tiles draws at most ceil(n_ctas * t / t_all) CTAs: keep that within kMaxHome
+    const long long home_cap = (long long)(kMaxHome - 1) * t_all / t_max;
+    const int n_ctas = (int)std::max<long long>(1, std::min<long long>(std::min<long long>(n_ctas_max, t_all / 2), home_cap));
     cta_unit0.assign(n_ctas, 0);
     cta_head0.assign(n_ctas, 0);
     cta_headn.assign(n_ctas, 0);
@@ -154,6 +166,14 @@ int build_start_table(int units, int budget, const int32_t* unit_lens, int n_cta
             cta_headn[cta] = kHeadTiles;
             next0[u] += kHeadTiles;
         }
+    }
+    std::vector<int> home(U, 0);
+    for (int cta = 0; cta < n_ctas; ++cta) home[cta_unit0[cta]] += 1;
+    chunk.assign(U, 2);
+    for (int u = 0; u < U; ++u) {
+        const int pulls = kMaxParts - 8 - std::min(home[u], kMaxHome);     // >= 24
+        const int t = (int)(tile_begin[u + 1] - tile_begin[u]) - next0[u]; // tiles the counter hands out
+        chunk[u] = std::max(2, ceil_div(std::max(t, 1), pulls));
     }
     return n_ctas;
 }
@@ -206,6 +226,7 @@ LayerDev layer_dev(const mkv_ctx* c, int layer) {
     d.cta_headn = (const int32_t*)(base + o.cta_headn);
     d.unit_lp = (const int32_t*)(base + o.unit_lp);
     d.unit_next0 = (const int32_t*)(base + o.unit_next0);
+    d.unit_chunk = (const int32_t*)(base + o.unit_chunk);
     d.next = (int32_t*)(base + o.next);
     d.cnt = (int2*)(base + o.cnt);
     d.launch_no = (uint32_t*)(base + o.launch_no);
@@ -276,20 +297,21 @@ size_t mkv_workspace_bytes(int layers, int batch, int q_heads, int kv_heads, int
 
 mkv_status mkv_plan_starts(int batch, int kv_heads, int budget, const int32_t* prefill_lens, int n_ctas_max,
                            int32_t* n_ctas, int32_t* cta_unit0, int32_t* cta_head0, int32_t* cta_headn,
-                           int32_t* unit_next0) {
+                           int32_t* unit_next0, int32_t* unit_chunk) {
     if (batch < 1 || kv_heads < 1 || budget < 1 || !prefill_lens || n_ctas_max < 1 || n_ctas_max > kMaxCtas)
         return MKV_ERR_INVALID_ARG;
-    if (!n_ctas || !cta_unit0 || !cta_head0 || !cta_headn || !unit_next0) return MKV_ERR_INVALID_ARG;
+    if (!n_ctas || !cta_unit0 || !cta_head0 || !cta_headn || !unit_next0 || !unit_chunk) return MKV_ERR_INVALID_ARG;
     for (int b = 0; b < batch; ++b)
         if (prefill_lens[b] < 0) return MKV_ERR_INVALID_ARG;
-    std::vector<int32_t> lp, next0, u0, h0, hn, ul((size_t)batch * kv_heads);
+    std::vector<int32_t> lp, next0, ch, u0, h0, hn, ul((size_t)batch * kv_heads);
     for (size_t u = 0; u < ul.size(); ++u) ul[u] = prefill_lens[u / kv_heads];
-    const int n = build_start_table(batch * kv_heads, budget, ul.data(), n_ctas_max, lp, next0, u0, h0, hn);
+    const int n = build_start_table(batch * kv_heads, budget, ul.data(), n_ctas_max, lp, next0, ch, u0, h0, hn);
     *n_ctas = n;
     std::memcpy(cta_unit0, u0.data(), sizeof(int32_t) * (size_t)n);
     std::memcpy(cta_head0, h0.data(), sizeof(int32_t) * (size_t)n);
     std::memcpy(cta_headn, hn.data(), sizeof(int32_t) * (size_t)n);
     std::memcpy(unit_next0, next0.data(), sizeof(int32_t) * next0.size());
+    std::memcpy(unit_chunk, ch.data(), sizeof(int32_t) * ch.size());
     return MKV_OK;
 }
 
@@ -385,8 +407,8 @@ mkv_status mkv_prefill_units(mkv_ctx* c, int layer, const void* K, const void* V
     const Layout& L = c->lay;
     const int U = L.units;
 
-    std::vector<int32_t> lp, next0, cta_unit0, cta_head0, cta_headn;
-    const int n_ctas = build_start_table(U, c->budget_max, unit_lens, c->n_ctas_max, lp, next0,
+    std::vector<int32_t> lp, next0, chunk, cta_unit0, cta_head0, cta_headn;
+    const int n_ctas = build_start_table(U, c->budget_max, unit_lens, c->n_ctas_max, lp, next0, chunk,
                                          cta_unit0, cta_head0, cta_headn);
     c->n_ctas[layer] = n_ctas;
     for (int u = 0; u < U; ++u) c->lens[layer][u] = unit_lens[u];
@@ -398,6 +420,7 @@ mkv_status mkv_prefill_units(mkv_ctx* c, int layer, const void* K, const void* V
     ok &= cudaMemcpyAsync(base + L.lo.cta_headn, cta_headn.data(), (size_t)n_ctas * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok &= cudaMemcpyAsync(base + L.lo.unit_lp, lp.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok &= cudaMemcpyAsync(base + L.lo.unit_next0, next0.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(base + L.lo.unit_chunk, chunk.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok &= cudaMemcpyAsync(base + L.lo.next, next0.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok &= cudaMemcpyAsync(base + L.lo.next + (size_t)U * 4, next0.data(), U * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok &= cudaMemsetAsync(base + L.lo.cnt, 0, 2 * (size_t)U * 8, st) == cudaSuccess;

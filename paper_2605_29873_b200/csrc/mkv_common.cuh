@@ -48,6 +48,7 @@ constexpr int kMaxGroup = 8;        // G = q_heads / kv_heads the kernels are bu
 constexpr int kMaxParts = 64;       // partials per unit (chunks grow to keep this)
 constexpr int kMaxCtas = 2048;      // persistent grid upper bound
 constexpr int kHeadTiles = 3;       // tiles a CTA owns outright at its starting place
+constexpr int kMaxHome = 32;        // CTAs that start in one unit (bound kept by the start table)
 constexpr float kNegBig = -1.0e30f; // finite stand-in for -inf in running maxima
 
 enum : int { kModeDecode = 0, kModeAttendOnly = 1 };
@@ -72,6 +73,7 @@ struct LayerDev {
     const int32_t* cta_headn;   // [n_ctas] number of reserved tiles (prefill tiles; may be 0)
     const int32_t* unit_lp;     // [units] prefill length
     const int32_t* unit_next0;  // [units] tiles reserved in the unit = start value of its counter
+    const int32_t* unit_chunk;  // [units] tiles handed out per pull of the unit's counter
     // Work-sharing counters, two copies each (copy c at + c * n_units).  A launch uses the copy
     // of its own parity and its tails rewind the other one for the launch after it.  The parity
     // is found on the device: every CTA keeps, in a word of its own, the number of launches it
@@ -139,7 +141,6 @@ __device__ inline void bar_sync(int id, int nthreads) {
 __device__ inline int unit_tiles(int lp, int n_old) {
     return max(1, (lp + kTileRows - 1) / kTileRows + (n_old + kTileRows - 1) / kTileRows);
 }
-__device__ inline int unit_chunk(int total) { return max(2, (total + kMaxParts - 9) / (kMaxParts - 8)); }
 
 // Optional per-CTA timestamps (diagnostic builds only: compile with -DMKV_TRACE).  Slot i of
 // CTA c is g_trace[(launch parity * kMaxCtas + c) * 16 + i]; mkv_debug_trace() copies the array

@@ -303,7 +303,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         int32_t* const nxt = L.next + (size_t)par * L.n_units;
         int2* const cnt = L.cnt + (size_t)par * L.n_units;
         int total = unit_tiles(lp, n_old);
-        int chunk = unit_chunk(total);
+        int chunk = L.unit_chunk[u];
         if (lane == 0 && ok && has_head) {
             slot = atomicAdd(&cnt[u].y, 1);
             for (; head_t < head_end && ok; ++head_t) {
@@ -351,10 +351,11 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             int found = -1;
             for (int base = 1; base < U && found < 0; base += 32) {
                 const int k = base + lane;
-                int lpc = 0, ndc = 0, rem = 0;
+                int lpc = 0, ndc = 0, rem = 0, chc = 2;
                 if (k < U) {
                     const int cand = (u + k) % U;
                     lpc = L.unit_lp[cand];
+                    chc = L.unit_chunk[cand];
                     ndc = min(L.n_dec[cand], p.cap - (dec ? 1 : 0));
                     rem = max(0, unit_tiles(lpc, ndc) - __ldcg(&nxt[cand]));
                 }
@@ -368,12 +369,12 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
                     found = (u + base + src) % U;
                     lp = __shfl_sync(0xffffffffu, lpc, src);
                     n_old = __shfl_sync(0xffffffffu, ndc, src);
+                    chunk = __shfl_sync(0xffffffffu, chc, src);
                 }
             }
             if (found < 0) break;
             u = found;
             total = unit_tiles(lp, n_old);
-            chunk = unit_chunk(total);
             if (lane == 0) g = atomicAdd(&nxt[u], chunk);
         }
         if (lane == 0) {

@@ -74,7 +74,7 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
             if (tid == 0) atomicCAS(p.status, kStatusOk, kStatusDeviceCheck);
             n_old = p.cap - (dec ? 1 : 0);
         }
-        const int total = unit_tiles(lp, n_old), chunk = unit_chunk(total);
+        const int total = unit_tiles(lp, n_old), chunk = L.unit_chunk[u];
         float qf[G][EPL];
         {
             const T* qp = reinterpret_cast<const T*>(p.q) + ((size_t)b * p.q_heads + (size_t)g * G) * D + lane * EPL;

@@ -70,7 +70,7 @@ def load_library(path: str | None = None):
     L.mkv_read_kv.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, i32p, vp, vp, C.c_int]
     L.mkv_get_step.argtypes = [vp, C.c_int, C.POINTER(C.c_int64)]
     L.mkv_attend_noalloc.argtypes = [vp, vp, vp, vp] + [C.c_int] * 9 + [vp]
-    L.mkv_plan_starts.argtypes = [C.c_int, C.c_int, C.c_int, i32p, C.c_int, i32p, i32p, i32p, i32p, i32p]
+    L.mkv_plan_starts.argtypes = [C.c_int, C.c_int, C.c_int, i32p, C.c_int, i32p, i32p, i32p, i32p, i32p, i32p]
     L.mkv_status_string.restype = C.c_char_p
     L.mkv_status_string.argtypes = [C.c_int]
     if path is None:
@@ -113,16 +113,17 @@ def attend_noalloc(q, K, V, out, n_tokens, stream=None):
 
 def plan_starts(batch, kv_heads, budget, prefill_lens, n_ctas_max):
     """The kernels' start table for these lengths (``mkv_plan_starts``; host arithmetic only).
-    Returns (cta_unit0, cta_head0, cta_headn, unit_next0) as int32 arrays."""
+    Returns (cta_unit0, cta_head0, cta_headn, unit_next0, unit_chunk) as int32 arrays."""
     lens = np.ascontiguousarray(prefill_lens, dtype=np.int32)
     assert lens.shape == (batch,)
     n = C.c_int32(0)
     u0, h0, hn = (np.zeros(n_ctas_max, dtype=np.int32) for _ in range(3))
     nx = np.zeros(batch * kv_heads, dtype=np.int32)
+    ch = np.zeros(batch * kv_heads, dtype=np.int32)
     p = lambda a: a.ctypes.data_as(C.POINTER(C.c_int32))
     _check(load_library().mkv_plan_starts(batch, kv_heads, budget, p(lens), n_ctas_max, C.byref(n), p(u0), p(h0), p(hn),
-                                          p(nx)), "mkv_plan_starts")
-    return u0[: n.value].copy(), h0[: n.value].copy(), hn[: n.value].copy(), nx
+                                          p(nx), p(ch)), "mkv_plan_starts")
+    return u0[: n.value].copy(), h0[: n.value].copy(), hn[: n.value].copy(), nx, ch
 
 
 def _check(code, where):

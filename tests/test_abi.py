@@ -87,15 +87,17 @@ def test_create_validates_then_fails_loudly_without_a_gpu(lib):
 
 def test_start_table_invariants(lib):
     """mkv_plan_starts: CTAs are spread over the units in tile order, reserved tiles are
-    disjoint prefill tiles, and a unit's counter starts right behind them."""
+    disjoint prefill tiles, a unit's counter starts right behind them, and the CTAs starting in
+    a unit plus the pulls of its counter fit the 64 partial results a unit has room for."""
     import numpy as np
     from workloads.synthetic import CONFIGS
     cases = [(CONFIGS["llama_b16"].prefill_lens(), 8, 1024, 296), (np.array([64], dtype=np.int32), 1, 64, 296),
              (np.array([0, 5, 4096], dtype=np.int32), 4, 128, 296), (np.full(64, 512, dtype=np.int32), 4, 2048, 296),
-             (np.array([100000], dtype=np.int32), 2, 16, 7)]
+             (np.array([100000], dtype=np.int32), 2, 16, 7), (np.array([100000], dtype=np.int32), 2, 16, 296),
+             (np.array([30000, 100, 100, 50000], dtype=np.int32), 1, 4096, 2048)]
     for lens, hkv, budget, nmax in cases:
         B = len(lens)
-        u0, h0, hn, nx = mkv.plan_starts(B, hkv, budget, lens, nmax)
+        u0, h0, hn, nx, ch = mkv.plan_starts(B, hkv, budget, lens, nmax)
         U = B * hkv
         tiles = np.array([-(-int(lens[u // hkv]) // 64) + -(-budget // 64) for u in range(U)])
         assert 1 <= len(u0) <= nmax and len(u0) <= max(1, tiles.sum() // 2)
@@ -112,3 +114,5 @@ def test_start_table_invariants(lib):
             # reserved ranges tile [0, next0) without gaps, all inside the prefill tiles
             assert [g[0] for g in got] == list(range(0, 3 * len(got), 3))
             assert nx[u] == 3 * len(got) <= -(-int(lens[u // hkv]) // 64)
+            assert len(mine) <= 32 and ch[u] >= 2
+            assert len(mine) + -(-int(tiles[u] - nx[u]) // int(ch[u])) <= 64 - 8

@@ -68,6 +68,16 @@ def test_ragged_batch_bf16():
     assert rep.evicted_not_newest > 50
 
 
+def test_few_long_units_share_many_ctas():
+    """One sequence with a long prompt: eight units of ~320 tiles draw the whole grid, about 31
+    CTAs each, and every visit of a unit delivers one partial result; the start table must keep
+    visits within the room a unit has for them (no device-check status, results as the oracle's)."""
+    w = CONFIGS["llama_b1"].with_(prefill=20000, steps=45, budget=30, variant="hot", n_heavy=2)
+    rep = run_case(w, w.steps, check_every=5)
+    assert rep.ok(), rep.failures[:5]
+    assert rep.max_out_err <= 2e-3 and rep.max_score_err <= 1e-4
+
+
 def test_qwen_group7_bf16():
     """GQA group 7 (28 query heads on 4 KV heads): the padded head rows of the tensor-core
     kernel and the 8-head staging of the tail."""
