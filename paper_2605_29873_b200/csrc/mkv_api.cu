@@ -122,6 +122,8 @@ __global__ void prefill_copy_kernel(const uint8_t* __restrict__ srcK, const uint
     }
 }
 
+int g_min_chunk = 2;   // tiles per pull of a unit's counter, lower bound (MKV_MIN_CHUNK overrides, for tuning)
+
 // Start table.  A unit's rows are a sequence of 64-row tiles (prefill tiles, then decode
 // tiles); the CTAs are spread over the units in proportion to the units' tile counts (a
 // full decode pool assumed).  Each CTA owns kHeadTiles tiles outright at its place, if the
@@ -173,7 +175,7 @@ int build_start_table(int units, int budget, const int32_t* unit_lens, int n_cta
     for (int u = 0; u < U; ++u) {
         const int pulls = kMaxParts - 8 - std::min(home[u], kMaxHome);     // >= 24
         const int t = (int)(tile_begin[u + 1] - tile_begin[u]) - next0[u]; // tiles the counter hands out
-        chunk[u] = std::max(2, ceil_div(std::max(t, 1), pulls));
+        chunk[u] = std::max(g_min_chunk, ceil_div(std::max(t, 1), pulls));
     }
     return n_ctas;
 }
@@ -369,6 +371,7 @@ mkv_status mkv_create(int layers, int q_heads, int kv_heads, int head_dim, int b
     c->stepped.assign(layers, 0);
     c->pdl = true;
     if (const char* e = std::getenv("MKV_NO_OVERLAP")) c->pdl = std::atoi(e) == 0;
+    if (const char* e = std::getenv("MKV_MIN_CHUNK")) g_min_chunk = std::max(1, std::min(64, std::atoi(e)));
     c->n_ctas.assign(layers, 0);
     c->lens.assign(layers, std::vector<int32_t>((size_t)batch * kv_heads, 0));
     c->launches = 0;

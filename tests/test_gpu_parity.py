@@ -78,6 +78,31 @@ def test_few_long_units_share_many_ctas():
     assert rep.max_out_err <= 2e-3 and rep.max_score_err <= 1e-4
 
 
+def test_headline_sequences_through_ramp_and_steady_state():
+    """Two sequences of the headline workload at its real sizes (prefill 654 and 926 tokens of the
+    U[512,4096] draw, budget 1024, bf16), free-running against the oracle from the empty pool
+    through the whole ramp and 160 evicting steps: drift of the scores over more than a thousand
+    steps of Eq. 5 and every eviction at the full budget."""
+    w = CONFIGS["llama_b16"].with_(variant="hot")
+    rep = run_case(w, w.budget + 160, sequences=[9, 8], check_every=16)
+    assert rep.ok(), rep.failures[:5]
+    assert rep.max_out_err <= 2e-3 and rep.max_score_err <= 1e-4
+    assert rep.evictions == 2 * w.kv_heads * 160
+
+
+@pytest.mark.parametrize("budget,beta", [(128, 0.8), (128, 0.99), (512, 0.8), (512, 0.99)])
+def test_qwen_sweep_cells_one_sequence(budget, beta):
+    """Cells of the G=7 sweep at their real sizes (28/4 heads, prefill 512, the cell's budget and
+    momentum factor), one sequence each, free-running through the ramp and 100 evicting steps.
+    beta only enters Eq. 5, so the cells differ in how fast old attention fades: 0.99 keeps
+    scores of very different ages close together, 0.8 forgets within a few steps."""
+    w = CONFIGS["qwen_b64"].with_(budget=budget, beta=beta, variant="hot")
+    rep = run_case(w, budget + 100, sequences=[3], check_every=8)
+    assert rep.ok(), rep.failures[:5]
+    assert rep.max_out_err <= 2e-3 and rep.max_score_err <= 1e-4
+    assert rep.evictions == w.kv_heads * 100
+
+
 def test_qwen_group7_bf16():
     """GQA group 7 (28 query heads on 4 KV heads): the padded head rows of the tensor-core
     kernel and the 8-head staging of the tail."""
