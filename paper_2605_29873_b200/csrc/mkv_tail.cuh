@@ -255,20 +255,30 @@ __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB
     if (tid == 0) MKV_TR(10);
 
     // ---- 1. combine -----------------------------------------------------------------------
-    if (tid < G) {
-        float M = dec ? sm.snew[tid] : kNegBig;
-        for (int q = 0; q < P; ++q) M = fmaxf(M, sm.w[q][tid]);
-        float Lsum = 0.f;
-        for (int q = 0; q < P; ++q) {
-            const float w = fast_exp2(sm.w[q][tid] - M);
-            sm.w[q][tid] = w;
-            Lsum = fmaf(sm.pl[q][tid], w, Lsum);
+    // heads over the warps, partials over the lanes (two per lane: kMaxParts = 64)
+    static_assert(kMaxParts <= 64, "two partials per lane");
+    for (int h = warp; h < G; h += NW) {
+        const bool has0 = lane < P, has1 = lane + 32 < P;
+        const float m0 = has0 ? sm.w[lane][h] : kNegBig;
+        const float m1 = has1 ? sm.w[lane + 32][h] : kNegBig;
+        float M = fmaxf(m0, m1);
+        if (dec) M = fmaxf(M, sm.snew[h]);
+#pragma unroll
+        for (int off = 16; off; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+        const float w0 = has0 ? fast_exp2(m0 - M) : 0.f;
+        const float w1 = has1 ? fast_exp2(m1 - M) : 0.f;
+        float Lsum = (has0 ? sm.pl[lane][h] * w0 : 0.f) + (has1 ? sm.pl[lane + 32][h] * w1 : 0.f);
+#pragma unroll
+        for (int off = 16; off; off >>= 1) Lsum += __shfl_xor_sync(0xffffffffu, Lsum, off);
+        if (has0) sm.w[lane][h] = w0;
+        if (has1) sm.w[lane + 32][h] = w1;
+        if (lane == 0) {
+            float wn = 0.f;
+            if (dec) { wn = fast_exp2(sm.snew[h] - M); Lsum += wn; }
+            sm.wnew[h] = wn;
+            sm.M[h] = M;
+            sm.invL[h] = Lsum > 0.f ? 1.0f / Lsum : 0.f;
         }
-        float wn = 0.f;
-        if (dec) { wn = fast_exp2(sm.snew[tid] - M); Lsum += wn; }
-        sm.wnew[tid] = wn;
-        sm.M[tid] = M;
-        sm.invL[tid] = Lsum > 0.f ? 1.0f / Lsum : 0.f;
     }
     bar_sync(BAR, NT);
     // out, part 1: the fresh token and the partials staged in registers
