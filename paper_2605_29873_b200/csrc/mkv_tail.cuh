@@ -205,7 +205,7 @@ __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB
     const int lane = tid & 31, warp = tid >> 5;
     constexpr int NW = NT / 32;
     constexpr int TW = TailPre<NT, GB>::TW;
-    constexpr int PB = GB <= 4 ? 2 : 1;                 // partials staged in registers up front
+    constexpr int PB = GB <= 4 ? 4 : 1;                 // partials staged in registers up front
     constexpr int LB = 4;                               // partials fetched per trip after those
     constexpr int OCB = TailPre<NT, GB>::OCB;
     const T* knew = reinterpret_cast<const T*>(p.k_new) + (size_t)u * D;
