@@ -199,6 +199,7 @@ struct mkv_ctx {
     std::vector<int> n_ctas;
     std::vector<std::vector<int32_t>> lens;   // per layer, per (sequence, KV head) unit
     int64_t launches;
+    bool direct_out;   // mkv_decode_step_host may let the kernel write pinned host memory (MKV_NO_DIRECT_OUT=1: never)
 };
 
 namespace {
@@ -371,6 +372,8 @@ mkv_status mkv_create(int layers, int q_heads, int kv_heads, int head_dim, int b
     c->stepped.assign(layers, 0);
     c->pdl = true;
     if (const char* e = std::getenv("MKV_NO_OVERLAP")) c->pdl = std::atoi(e) == 0;
+    c->direct_out = true;
+    if (const char* e = std::getenv("MKV_NO_DIRECT_OUT")) c->direct_out = std::atoi(e) == 0;
     if (const char* e = std::getenv("MKV_MIN_CHUNK")) g_min_chunk = std::max(1, std::min(64, std::atoi(e)));
     c->n_ctas.assign(layers, 0);
     c->lens.assign(layers, std::vector<int32_t>((size_t)batch * kv_heads, 0));
@@ -485,10 +488,25 @@ mkv_status mkv_decode_step_host(mkv_ctx* c, int layer, const void* qh, const voi
         if (cudaMemcpyAsync(dk, kh, nk * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return MKV_ERR_CUDA;
         if (cudaMemcpyAsync(dv, vh, nk * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return MKV_ERR_CUDA;
     }
-    const Params p = make_params(c, layer, dq, dk, dv, dout, kModeDecode);
+    // Pinned host memory is visible to the GPU through the unified address space: the kernel
+    // then writes `out` there itself (posted writes over the bus, complete when the kernel is)
+    // and the step needs one copy operation fewer.  Pageable memory takes the staged copy.
+    // (Asked on every call: an address can change hands between calls.)
+    void* direct = nullptr;
+    if (c->direct_out) {
+        cudaPointerAttributes at;
+        if (cudaPointerGetAttributes(&at, outh) == cudaSuccess) {
+            if (at.type == cudaMemoryTypeHost && at.devicePointer && aligned16(at.devicePointer)) direct = at.devicePointer;
+        } else {
+            cudaGetLastError();   // not a pointer the runtime knows: treat as pageable
+        }
+    }
+    void* const kernel_out = direct ? direct : (void*)dout;
+    const Params p = make_params(c, layer, dq, dk, dv, kernel_out, kModeDecode);
     const mkv_status s = launch_step(c, layer, p, st);
     if (s != MKV_OK) return s;
-    if (cudaMemcpyAsync(outh, dout, nq * os, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MKV_ERR_CUDA;
+    if (!direct && cudaMemcpyAsync(outh, dout, nq * os, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return MKV_ERR_CUDA;
     return MKV_OK;
 }
 

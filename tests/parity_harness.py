@@ -73,7 +73,7 @@ def prefill_both(ctx, w: Workload, stream: BatchStream, layer=0, mode=O.GROUP_ME
 
 
 def lockstep(ctx, w: Workload, stream: BatchStream, oracles, steps, layer=0, report: ParityReport | None = None,
-             check_state_every=1, chunk=64, host_api=False, host_packed=False):
+             check_state_every=1, chunk=64, host_api=False, host_packed=False, host_pinned=True):
     """Runs `steps` decode steps on both sides, comparing as described in the module doc."""
     torch = ctx.torch
     rep = report or ParityReport()
@@ -86,17 +86,18 @@ def lockstep(ctx, w: Workload, stream: BatchStream, oracles, steps, layer=0, rep
         nb = min(chunk, steps - done)
         qs, ks, vs = stream.next(nb)
         if host_api:
-            qd = to_device(qs, torch, dt, "cpu").pin_memory()
-            kd = to_device(ks, torch, dt, "cpu").pin_memory()
-            vd = to_device(vs, torch, dt, "cpu").pin_memory()
+            pin = (lambda t: t.pin_memory()) if host_pinned else (lambda t: t)   # pageable: the staged path
+            qd = pin(to_device(qs, torch, dt, "cpu"))
+            kd = pin(to_device(ks, torch, dt, "cpu"))
+            vd = pin(to_device(vs, torch, dt, "cpu"))
             if host_packed:      # q | k_new | v_new of a step back to back: the single-copy path
                 nq, nk = qd[0].numel(), kd[0].numel()
-                pk = torch.empty((nb, nq + 2 * nk), dtype=dt).pin_memory()
+                pk = pin(torch.empty((nb, nq + 2 * nk), dtype=dt))
                 pk[:, :nq] = qd.reshape(nb, -1); pk[:, nq:nq + nk] = kd.reshape(nb, -1); pk[:, nq + nk:] = vd.reshape(nb, -1)
                 qd = [pk[j, :nq] for j in range(nb)]
                 kd = [pk[j, nq:nq + nk] for j in range(nb)]
                 vd = [pk[j, nq + nk:] for j in range(nb)]
-            out_h = torch.zeros((B, w.q_heads, w.head_dim), dtype=odt).pin_memory()
+            out_h = pin(torch.zeros((B, w.q_heads, w.head_dim), dtype=odt))
         else:
             qd, kd, vd = (to_device(a, torch, dt, ctx.device) for a in (qs, ks, vs))
         for i in range(nb):

@@ -115,13 +115,16 @@ def test_qwen_group7_bf16():
 
 def test_empty_prefill_and_bf16_out_through_host_api():
     """No prompt at all (the decode pool is the whole cache), bf16 output, host-buffer entry
-    point: covers the unit with nothing cached at the first step."""
+    point: covers the unit with nothing cached at the first step.  The host buffers are pinned
+    (the kernel writes `out` into them directly), then pinned and packed (one input copy), then
+    pageable (staged copies both ways)."""
     w = CONFIGS["llama_b1"].with_(prefill=0, steps=150, budget=40, variant="hot", n_heavy=2)
     ctx = make_context(w, out_f32=False)
     stream = BatchStream(w, 0)
     oracles, _ = prefill_both(ctx, w, stream)
-    rep = lockstep(ctx, w, stream, oracles, 100, host_api=True)
-    rep = lockstep(ctx, w, stream, oracles, w.steps - 100, host_api=True, host_packed=True, report=rep)
+    rep = lockstep(ctx, w, stream, oracles, 70, host_api=True)
+    rep = lockstep(ctx, w, stream, oracles, 40, host_api=True, host_packed=True, report=rep)
+    rep = lockstep(ctx, w, stream, oracles, w.steps - 110, host_api=True, host_pinned=False, report=rep)
     ctx.close()
     assert rep.ok(), rep.failures[:5]
     assert rep.evictions == (w.steps - w.budget) * w.kv_heads
