@@ -460,7 +460,7 @@ def main():
             line["e2e"] = {"value": world * B / (ms_e2e_max * 1e-3), "unit": "tokens/s",
                            "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                            "ms_per_step": ms_e2e_max, "sync": "stream synchronised after every step",
-                           "how": "one pinned host->device copy of q|k_new|v_new per step; the kernel writes out into the pinned host buffer"}
+                           "how": "per step the GPU fetches q|k_new|v_new from the pinned host buffer (a small kernel ahead of the step) and the step's kernel writes out into the pinned host buffer"}
         if not args.no_cpu_baseline and world == 1:
             n_units = min(len(os.sched_getaffinity(0)), B * Hkv)
             v, threads, sample, _ = time_oracle(w, lens, n_units, steps=48, warmup=2, time_cap_s=40.0, min_time_s=12.0)

@@ -188,9 +188,11 @@ mkv_status mkv_decode_step(mkv_ctx* ctx, int layer, const void* q, const void* k
  * Same step with HOST buffers: copies q, k_new, v_new to the device, runs the step,
  * copies `out` back; all on `stream`, asynchronous when the host buffers are pinned
  * (the caller synchronises the stream before reading `out` or reusing the inputs).  When
- * q, k_new and v_new lie back to back in host memory they travel as one copy.  An `out`
- * buffer in pinned, 16-byte aligned host memory is written by the kernel directly instead
- * of by a copy after it; either way it is complete once the stream has been synchronised.
+ * q, k_new and v_new lie back to back in host memory they travel as one copy.  Pinned,
+ * 16-byte aligned host buffers are reached by the GPU in place: the inputs are fetched by a
+ * small kernel ahead of the step and `out` is written by the step's kernel itself, instead
+ * of copy operations before and after it; pageable buffers take staged copies.  Either way
+ * `out` is complete once the stream has been synchronised.
  */
 mkv_status mkv_decode_step_host(mkv_ctx* ctx, int layer, const void* q_host, const void* k_new_host,
                                 const void* v_new_host, void* out_host, void* stream);

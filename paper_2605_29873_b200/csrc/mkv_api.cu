@@ -10,6 +10,7 @@
 
 #include "../../include/mkv.h"
 #include "mkv_launch.h"
+#include "mkv_ptx.cuh"
 
 using namespace mkv;
 
@@ -123,6 +124,35 @@ __global__ void prefill_copy_kernel(const uint8_t* __restrict__ srcK, const uint
 }
 
 int g_min_chunk = 2;   // tiles per pull of a unit's counter, lower bound (MKV_MIN_CHUNK overrides, for tuning)
+
+// The step's inputs from pinned host memory into the staging area, read over the bus by the
+// GPU itself (16 bytes per thread).  Cheaper to start than a copy operation, and the step's
+// kernel, launched right behind with programmatic serialization, may begin its own start-up
+// meanwhile: it waits for this grid before it reads the staging area.
+struct HostPiece { const uint4* src; uint4* dst; int n16; };
+__global__ void host_gather_kernel(const HostPiece a, const HostPiece b, const HostPiece c3) {
+    ptx::griddep_launch_dependents();
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < a.n16) { a.dst[i] = a.src[i]; return; }
+    i -= a.n16;
+    if (i < b.n16) { b.dst[i] = b.src[i]; return; }
+    i -= b.n16;
+    if (i < c3.n16) c3.dst[i] = c3.src[i];
+}
+
+// The device's view of pinned host memory [p, p + bytes), or nullptr if the GPU cannot read it
+// in place (pageable memory, unknown pointer, not 16-byte aligned).
+void* pinned_view(const void* p, size_t bytes) {
+    cudaPointerAttributes a0, a1;
+    if (cudaPointerGetAttributes(&a0, p) != cudaSuccess ||
+        cudaPointerGetAttributes(&a1, (const uint8_t*)p + bytes - 1) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    if (a0.type != cudaMemoryTypeHost || a1.type != cudaMemoryTypeHost || !a0.devicePointer || !a1.devicePointer) return nullptr;
+    if ((const uint8_t*)a1.devicePointer - (const uint8_t*)a0.devicePointer != (ptrdiff_t)(bytes - 1)) return nullptr;
+    return ((uintptr_t)a0.devicePointer & 15u) == 0 ? a0.devicePointer : nullptr;
+}
 
 // Start table.  A unit's rows are a sequence of 64-row tiles (prefill tiles, then decode
 // tiles); the CTAs are spread over the units in proportion to the units' tile counts (a
@@ -477,7 +507,30 @@ mkv_status mkv_decode_step_host(mkv_ctx* c, int layer, const void* qh, const voi
     uint8_t *dq = c->ws + c->lay.stage_q, *dk = c->ws + c->lay.stage_k, *dv = c->ws + c->lay.stage_v,
             *dout = c->ws + c->lay.stage_out;
     const uint8_t* q8 = (const uint8_t*)qh;
-    if ((const uint8_t*)kh == q8 + nq * es && (const uint8_t*)vh == q8 + (nq + nk) * es) {
+    const bool packed = (const uint8_t*)kh == q8 + nq * es && (const uint8_t*)vh == q8 + (nq + nk) * es;
+    bool gathered = false;
+    if (c->direct_out && ((nq * es) | (nk * es)) % 16 == 0) {
+        // pinned inputs: the GPU fetches them itself (see host_gather_kernel)
+        HostPiece pq{nullptr, (uint4*)dq, (int)(nq * es / 16)}, pk{nullptr, (uint4*)dk, (int)(nk * es / 16)},
+            pv{nullptr, (uint4*)dv, (int)(nk * es / 16)};
+        if (packed) {
+            pq.src = (const uint4*)pinned_view(qh, (nq + 2 * nk) * es);
+            if (pq.src) { pk.src = pq.src + pq.n16; pv.src = pk.src + pk.n16; }
+        } else {
+            pq.src = (const uint4*)pinned_view(qh, nq * es);
+            pk.src = (const uint4*)pinned_view(kh, nk * es);
+            pv.src = (const uint4*)pinned_view(vh, nk * es);
+        }
+        if (pq.src && pk.src && pv.src) {
+            const int total = pq.n16 + pk.n16 + pv.n16, threads = 256;
+            host_gather_kernel<<<(total + threads - 1) / threads, threads, 0, st>>>(pq, pk, pv);
+            if (cudaGetLastError() != cudaSuccess) return MKV_ERR_CUDA;
+            c->launches += 1;
+            gathered = true;
+        }
+    }
+    if (gathered) {
+    } else if (packed) {
         // q, k_new and v_new lie back to back on the host: one copy instead of three (the three
         // staging regions are adjacent and at least as large)
         dk = dq + nq * es;
