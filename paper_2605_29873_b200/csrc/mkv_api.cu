@@ -530,6 +530,7 @@ mkv_status mkv_decode_step_host(mkv_ctx* c, int layer, const void* qh, const voi
         }
     }
     if (gathered) {
+        // nothing left to copy
     } else if (packed) {
         // q, k_new and v_new lie back to back on the host: one copy instead of three (the three
         // staging regions are adjacent and at least as large)
@@ -545,15 +546,7 @@ mkv_status mkv_decode_step_host(mkv_ctx* c, int layer, const void* qh, const voi
     // then writes `out` there itself (posted writes over the bus, complete when the kernel is)
     // and the step needs one copy operation fewer.  Pageable memory takes the staged copy.
     // (Asked on every call: an address can change hands between calls.)
-    void* direct = nullptr;
-    if (c->direct_out) {
-        cudaPointerAttributes at;
-        if (cudaPointerGetAttributes(&at, outh) == cudaSuccess) {
-            if (at.type == cudaMemoryTypeHost && at.devicePointer && aligned16(at.devicePointer)) direct = at.devicePointer;
-        } else {
-            cudaGetLastError();   // not a pointer the runtime knows: treat as pageable
-        }
-    }
+    void* const direct = c->direct_out ? pinned_view(outh, nq * os) : nullptr;
     void* const kernel_out = direct ? direct : (void*)dout;
     const Params p = make_params(c, layer, dq, dk, dv, kernel_out, kModeDecode);
     const mkv_status s = launch_step(c, layer, p, st);
