@@ -29,7 +29,7 @@ struct LayerOff {
 // Scratch that lives for one step only, shared by all layers of the context (calls on a
 // context are ordered on one stream, and a step touches it only after every earlier kernel
 // of the stream has completed).
-struct ScratchOff { size_t logit, part_o, part_ml, keys, list_a, list_b, end; };
+struct ScratchOff { size_t logit, head_sum, part_o, part_ml, keys, list_a, list_b, end; };
 struct Layout {
     int units, cap, rowb, lstride;
     size_t status, stage_q, stage_k, stage_v, stage_out, scratch0, scratch_bytes, layer0, layer_bytes, total;
@@ -62,6 +62,7 @@ bool make_layout(int layers, int batch, int q_heads, int kv_heads, int head_dim,
     const size_t U = (size_t)L.units, C = (size_t)L.cap;
     o = 0;
     L.so.logit = take((size_t)batch * q_heads * L.lstride * 4);
+    L.so.head_sum = take((size_t)batch * L.lstride * 4);   // zero from mkv_create's memset, kept zero by its users
     L.so.part_o = take(U * kMaxParts * G * head_dim * 4);
     L.so.part_ml = take(U * kMaxParts * G * 2 * 4);
     L.so.keys = take(U * C * 8);
@@ -246,6 +247,7 @@ LayerDev layer_dev(const mkv_ctx* c, int layer) {
     d.pos = (int32_t*)(base + o.pos);
     d.n_dec = (int32_t*)(base + o.n_dec);
     d.logit = (float*)(sb + so.logit);
+    d.head_sum = (float*)(sb + so.head_sum);
     d.abar = (c->flags & MKV_FLAG_RECORD_PROBS) ? (float*)(base + o.abar) : nullptr;
     d.abar_pos = (int32_t*)(base + o.abar_pos);
     d.n_prev = (int32_t*)(base + o.n_prev);

@@ -60,6 +60,8 @@ struct LayerDev {
     int32_t* pos;
     int32_t* n_dec;
     float* logit;      // [batch*q_heads][lstride] raw logits (log2 units) of decode-pool tokens
+    float* head_sum;   // [batch][lstride] layer-wide score mode: per decode token the probabilities summed over
+                       // all heads of the sequence (accumulated by its units' tails); all zero between steps
     float* abar;       // [units][cap] or nullptr: Eq. 4 values of the last step, slot order before its eviction
     int32_t* abar_pos; // [units][cap], with abar: the position ids of those slots
     int32_t* n_prev;   // [units] decode count (fresh token included) before the last eviction

@@ -4,10 +4,11 @@
 // head).  The streaming loops run unchanged.  When a (sequence, KV head) unit is complete its
 // tail does that head's share (unit_tail in its LAYER form):
 //   the fresh token's logits, the cross-split combine, `out`                        (Eq. 2)
-//   per decode token the sum over the unit's G heads of 2^(s - M_h) / L_h
+//   per decode token the sum over the unit's G heads of 2^(s - M_h) / L_h, added to the
+//   sequence's row of head sums
 // and the tail that finishes last for a sequence (a ticket) goes on with what needs all heads
 // (layer_finish, this file):
-//   per decode token: abar = (1/H) sum of those sums over the KV heads               (Eq. 4)
+//   per decode token: abar = (1/H) of the summed probabilities of all H heads         (Eq. 4)
 //   I <- beta * I + abar, the fresh token starting from 0                            (Eq. 5, 6)
 //   one selection of the overflow-many lowest (score bits, position id) keys         (Eq. 7, 8)
 //   the same append / hole filling in every KV head's pool                           (Eq. 9)
@@ -24,7 +25,6 @@ namespace mkv {
 template <typename T, int NT, int BAR, int GB>
 __device__ void layer_finish(const Params& p, int u, const TailPre<NT, GB>& pre, TailSmem<NT>& sm, int tid) {
     constexpr int NW = NT / 32;
-    constexpr int HB = 8;                              // KV heads fetched per trip
     constexpr int TW = TailPre<NT, GB>::TW;            // tokens per thread and pass
     const LayerDev& L = p.L;
     const int lane = tid & 31, warp = tid >> 5;
@@ -52,47 +52,33 @@ __device__ void layer_finish(const Params& p, int u, const TailPre<NT, GB>& pre,
     const int n = n_old + 1;
     const int t = pre.t;
     const int k = max(0, n - p.budget);
-    // row of KV head g2's sums: the first logit row of its unit
-    const float* sums = L.logit + (size_t)b * Hq * ls;
-    const size_t sum_stride = (size_t)G * ls;
+    // the sequence's head sums, complete now; this tail reads them and leaves the row at zero
+    float* const sums = L.head_sum + (size_t)b * ls;
 
     // ---- all heads: head mean, momentum update -----------------------------------------------
-    // Latency again: the fresh token's sums are fetched now and used after the loop.
     const float inv_h = 1.0f / (float)Hq;
-    float fresh[HB];
-#pragma unroll
-    for (int j = 0; j < HB; ++j) fresh[j] = j < Hkv ? __ldcg(sums + j * sum_stride + n_old) : 0.f;
+    const float ab_new = __ldcg(sums + n_old) * inv_h;     // Eq. 6: I_fresh = alpha * 0 + abar_fresh
+    const unsigned long long key_new = ((unsigned long long)__float_as_uint(ab_new) << 32) | (unsigned)t;
     unsigned long long* keys = L.keys + (size_t)u0 * cap;
     const float* score0 = L.score + (size_t)u0 * ls;
     const int32_t* pos0 = L.pos + (size_t)u0 * ls;
     unsigned long long best_key = ~0ull;
     int best_slot = -1;
-    // TW tokens per thread and pass; one batch of loads per pass (rows are lstride floats long,
-    // a multiple of 4, so whole vectors stay inside them)
-    for (int i0 = TW * tid; i0 < n_old; i0 += TW * NT) {
-        float s[TW];
-#pragma unroll
-        for (int j = 0; j < TW; ++j) s[j] = 0.f;
-        float sc[TW];
-        int ps[TW];
-        load_vec<TW>(score0 + i0, sc);
-        load_vec<TW>(pos0 + i0, ps);
-        for (int g0 = 0; g0 < Hkv; g0 += HB) {
-            float v[HB][TW];
-#pragma unroll
-            for (int j = 0; j < HB; ++j)
-                if (g0 + j < Hkv) load_vec<TW>(sums + (size_t)(g0 + j) * sum_stride + i0, v[j]);
-#pragma unroll
-            for (int j = 0; j < HB; ++j)
-                if (g0 + j < Hkv) {
-#pragma unroll
-                    for (int e = 0; e < TW; ++e) s[e] += v[j][e];
-                }
-        }
+    // TW tokens per thread and pass, two passes per trip: their loads are issued together (rows
+    // are lstride floats long, a multiple of 4, so whole vectors stay inside them)
+    auto token_pass = [&](int i0, const float (&s)[TW], const float (&sc)[TW], const int (&ps)[TW]) {
+        if (i0 >= n_old) return;
         float ab[TW], nw[TW];
 #pragma unroll
         for (int j = 0; j < TW; ++j) { ab[j] = s[j] * inv_h; nw[j] = fmaf(p.beta, sc[j], ab[j]); }
         const bool whole = i0 + TW <= n_old;
+        // slots below n_old go back to zero (slot n_old, which every thread reads above, later)
+        if (whole) {
+            if constexpr (TW == 4) *reinterpret_cast<float4*>(sums + i0) = make_float4(0.f, 0.f, 0.f, 0.f);
+            else *reinterpret_cast<float2*>(sums + i0) = make_float2(0.f, 0.f);
+        } else {
+            for (int j = 0; j < TW; ++j) if (i0 + j < n_old) sums[i0 + j] = 0.f;
+        }
         for (int g2 = 0; g2 < Hkv; ++g2) {
             float* sg = L.score + (size_t)(u0 + g2) * ls + i0;
             if (whole) {
@@ -116,14 +102,19 @@ __device__ void layer_finish(const Params& p, int u, const TailPre<NT, GB>& pre,
                 if (key < best_key) { best_key = key; best_slot = i0 + j; }
             }
         }
+    };
+    for (int base = 0; base < n_old; base += 2 * TW * NT) {
+        const int ia = base + TW * tid, ib = ia + TW * NT;
+        float sa[TW], sca[TW], sb[TW], scb[TW];
+        int psa[TW], psb[TW];
+        if (ia < n_old) { load_vec<TW>(sums + ia, sa); load_vec<TW>(score0 + ia, sca); load_vec<TW>(pos0 + ia, psa); }
+        if (ib < n_old) { load_vec<TW>(sums + ib, sb); load_vec<TW>(score0 + ib, scb); load_vec<TW>(pos0 + ib, psb); }
+        token_pass(ia, sa, sca, psa);
+        token_pass(ib, sb, scb, psb);
     }
-    float ab_new = 0.f;
-#pragma unroll
-    for (int j = 0; j < HB; ++j) ab_new += fresh[j];
-    for (int g2 = HB; g2 < Hkv; ++g2) ab_new += __ldcg(sums + g2 * sum_stride + n_old);
-    ab_new *= inv_h;                                   // Eq. 6: I_fresh = alpha * 0 + abar_fresh
-    const unsigned long long key_new = ((unsigned long long)__float_as_uint(ab_new) << 32) | (unsigned)t;
+    bar_sync(BAR, NT);                                 // every thread has read slot n_old
     if (tid == NT - 1) {                               // the fresh token sits (virtually) in slot n_old
+        sums[n_old] = 0.f;
         if (key_new < best_key) { best_key = key_new; best_slot = n_old; }
         if (L.abar)
             for (int g2 = 0; g2 < Hkv; ++g2) {
