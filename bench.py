@@ -346,14 +346,23 @@ def main():
     barrier()
     launches0 = ctx.launch_count()
     sampler.start()
+    # five equal segments of the timed region get events of their own (spread of the step time)
+    n_seg = 5 if args.steps >= 50 else 1
+    seg_ev = [torch.cuda.Event(enable_timing=True) for _ in range(n_seg - 1)]
+    seg_at = {args.steps * (j + 1) // n_seg: seg_ev[j] for j in range(n_seg - 1)}
     ev0.record(stream)
     for i in range(args.steps):
         step(i)
+        if i + 1 in seg_at:
+            seg_at[i + 1].record(stream)
     ev1.record(stream)
     barrier()
     clocks = sampler.stop()
     launches = ctx.launch_count() - launches0
     ms = ev0.elapsed_time(ev1)
+    marks = [ev0] + seg_ev + [ev1]
+    bounds = [0] + sorted(seg_at) + [args.steps]
+    seg_ms = [marks[j].elapsed_time(marks[j + 1]) / max(bounds[j + 1] - bounds[j], 1) for j in range(n_seg)]
     ctx.status_sync()
 
     # plain decode attention on the same state (no append/score/evict): overhead reference
@@ -453,6 +462,10 @@ def main():
         line["whole_run"] = {"steps_per_layer": T, "ms_per_step": run_ms / T,
                              "tokens_per_s": world * B * T / (run_ms * 1e-3),
                              "how": "measured ramp mean x fill steps + measured steady state x the rest"}
+        if world == 1:
+            srt = sorted(seg_ms)
+            line["segments"] = {"n": n_seg, "median_ms_per_step": srt[len(srt) // 2], "min_ms_per_step": srt[0],
+                                "max_ms_per_step": srt[-1]}
         if ms_graph_max > 0.0:
             line["graph_replay"] = {"ms_per_step": ms_graph_max, "steps_per_graph": n_rec,
                                     "tokens_per_s": world * B / (ms_graph_max * 1e-3)}
