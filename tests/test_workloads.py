@@ -38,3 +38,21 @@ def test_config_shapes_and_heavy_hitters():
     bs = BatchStream(CONFIGS["qwen_b64"].with_(batch=3, steps=4))
     q, k, v = bs.next(4)
     assert q.shape == (4, 3, 28, 128) and k.shape == (4, 3, 4, 128)
+
+
+def test_algorithmic_bytes_of_the_headline_step():
+    """The roofline numerator: K and V of every cached token once per KV head, the appended rows,
+    the scores read and written, q and out, and one row moved per unit -- 237.8 MB for the
+    headline workload, written out here term by term."""
+    import bench
+    w = CONFIGS["llama_b16"]
+    lens = w.prefill_lens()
+    assert int(lens.sum()) == 41292
+    n, units = w.budget + 1, w.batch * w.kv_heads
+    want = (w.kv_heads * (int(lens.sum()) + w.batch * n) * 512     # K+V rows streamed
+            + units * 512                                           # fresh rows appended
+            + units * n * 8                                         # scores read and written
+            + 2 * w.batch * w.q_heads * w.head_dim * 2              # q in, out back (bf16)
+            + units * 1 * 2 * 520)                                  # one token moved per unit
+    assert want == 237816832
+    assert bench.algorithmic_bytes_per_step(w, lens, n, 1) == want
