@@ -100,7 +100,7 @@ size_t mkv_workspace_bytes(int layers, int batch, int q_heads, int kv_heads, int
  * The start table mkv_prefill() builds for the kernels, as pure host arithmetic (for
  * inspection and tests).  The rows of a (sequence, KV head) unit form 64-row tiles, prefill
  * tiles first; CTAs are spread over the units in proportion to the units' tile counts and
- * each owns up to 3 reserved prefill tiles where it starts, the rest being handed out by
+ * each owns up to 4 reserved prefill tiles where it starts, the rest being handed out by
  * per-unit counters at run time, unit_chunk tiles per pull.  At most 32 CTAs start in one
  * unit (the grid shrinks when few, long units would draw more), and a unit's chunk is sized so
  * that the CTAs starting there plus the pulls of its counter stay within the 64 partial results
@@ -109,7 +109,7 @@ size_t mkv_workspace_bytes(int layers, int batch, int q_heads, int kv_heads, int
  *   n_ctas_max      upper bound of the grid (1..2048)
  *   n_ctas          host out: CTAs used
  *   cta_unit0/head0/headn   host out, [n_ctas_max]: unit a CTA starts in, its first reserved
- *                   tile there, and how many tiles it has reserved (0 or 3)
+ *                   tile there, and how many tiles it has reserved (0 or 4)
  *   unit_next0      host out, [batch*kv_heads]: reserved tiles per unit = start value of the
  *                   unit's counter
  *   unit_chunk      host out, [batch*kv_heads]: tiles per pull of the unit's counter (>= 2)

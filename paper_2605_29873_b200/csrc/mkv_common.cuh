@@ -47,7 +47,7 @@ constexpr int kTileRows = 64;       // rows of one tile of the work decompositio
 constexpr int kMaxGroup = 8;        // G = q_heads / kv_heads the kernels are built for
 constexpr int kMaxParts = 64;       // partials per unit (chunks grow to keep this)
 constexpr int kMaxCtas = 2048;      // persistent grid upper bound
-constexpr int kHeadTiles = 3;       // tiles a CTA owns outright at its starting place
+constexpr int kHeadTiles = 4;       // tiles a CTA owns outright at its starting place (the ring holds 3 before the wait)
 constexpr int kMaxHome = 32;        // CTAs that start in one unit (bound kept by the start table)
 constexpr float kNegBig = -1.0e30f; // finite stand-in for -inf in running maxima
 
