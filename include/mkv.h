@@ -37,6 +37,16 @@
  *     mkv_prefill*(), the *_host entry points and the mkv_get_*() readers synchronise or copy
  *     from pageable memory and cannot be recorded.  mkv_launch_count() counts enqueued
  *     kernels, not replays.
+ *   - The kernels are persistent: the CTAs of a launch hand work to one another and a unit's
+ *     finishing part waits (bounded) for tiles that other CTAs deliver, so all CTAs of a launch
+ *     must be resident at once.  mkv_create() sizes the grid from the occupancy the device
+ *     reports for the kernel (SM count x resident CTAs per SM, see mkv_grid_limit()), which
+ *     holds as long as the GPU's SMs are not shared with other work for the length of a step:
+ *     kernels of other streams or processes that occupy SMs meanwhile can delay a step up to
+ *     the wait limit (MKV_OPT_WAIT_LIMIT_US), after which it ends with MKV_ERR_TIMEOUT.
+ *   - Several layers per launch: the layers of a context are independent instances of
+ *     Algorithm 1, and mkv_decode_step_layers() steps a run of consecutive layers with one
+ *     kernel launch (inputs stacked by layer).  Small per-layer batches fill the GPU that way.
  */
 #ifndef MKV_H_
 #define MKV_H_
@@ -86,6 +96,39 @@ typedef enum {
 #define MKV_FLAG_RECORD_PROBS 1u /* keep the head-averaged decode probabilities of the last
                                     step (Eq. 4) and their position ids, for
                                     mkv_get_last_probs() and mkv_recency_diagnostics()  */
+#define MKV_FLAG_INPUTS_READY 2u /* a promise by the caller: q, k_new and v_new of every
+                                    mkv_decode_step*() / mkv_attend_only*() call are final in
+                                    device memory when the call is made -- nothing still pending
+                                    on any stream writes them.  A step may then begin its
+                                    attention over the frozen prompt rows while the previous
+                                    kernel of the stream (normally the previous step) is still
+                                    finishing.  Without the flag a step reads q only after every
+                                    earlier kernel of the stream has completed.  (The *_host
+                                    entry points ignore the flag.)                           */
+#define MKV_FLAG_REPRODUCIBLE 4u /* same inputs, same bits: work is split among the CTAs by a
+                                    fixed table instead of run-time counters and partial results
+                                    are combined in a fixed order.  Costs some load balance;
+                                    meant for debugging and for race hunting (two runs must
+                                    agree bit for bit).  Without it `out` and the scores can
+                                    differ in their last bits from run to run.               */
+
+/* options for mkv_set_option */
+typedef enum {
+    MKV_OPT_RING_STAGES = 1,   /* tensor-core kernel: stages of its shared-memory ring, 2..6
+                                  (default 3; 32 KB each).  The grid is re-sized from the
+                                  occupancy that results (4 or more stages leave room for one
+                                  CTA per SM instead of two).  Layers must be prefilled again. */
+    MKV_OPT_HEAD_TILES = 2,    /* 64-row prompt tiles a CTA owns outright where it starts, 0..16
+                                  (default 4): they are fetched, and with MKV_FLAG_INPUTS_READY
+                                  also attended, before the previous step has ended.  Layers
+                                  must be prefilled again.                                    */
+    MKV_OPT_WAIT_LIMIT_US = 3, /* limit of every wait inside a kernel, microseconds
+                                  (default 2,000,000); on expiry the step ends early and the
+                                  sticky status becomes MKV_ERR_TIMEOUT                       */
+    MKV_OPT_OVERLAP = 4        /* 1 (default): consecutive steps on a stream overlap their
+                                  start-up with the previous step's end (programmatic
+                                  dependent launch); 0: plain stream order                    */
+} mkv_option;
 
 /*
  * Size in bytes of the workspace mkv_create() needs for these parameters
@@ -100,7 +143,7 @@ size_t mkv_workspace_bytes(int layers, int batch, int q_heads, int kv_heads, int
  * The start table mkv_prefill() builds for the kernels, as pure host arithmetic (for
  * inspection and tests).  The rows of a (sequence, KV head) unit form 64-row tiles, prefill
  * tiles first; CTAs are spread over the units in proportion to the units' tile counts and
- * each owns up to 4 reserved prefill tiles where it starts, the rest being handed out by
+ * each owns up to head_tiles reserved prefill tiles where it starts, the rest being handed out by
  * per-unit counters at run time, unit_chunk tiles per pull.  At most 32 CTAs start in one
  * unit (the grid shrinks when few, long units would draw more), and a unit's chunk is sized so
  * that the CTAs starting there plus the pulls of its counter stay within the 64 partial results
@@ -108,15 +151,36 @@ size_t mkv_workspace_bytes(int layers, int batch, int q_heads, int kv_heads, int
  *   prefill_lens    host, [batch]
  *   n_ctas_max      upper bound of the grid (1..2048)
  *   n_ctas          host out: CTAs used
+ *   head_tiles      tiles a CTA reserves where it starts (0..16; the library's default is 4)
  *   cta_unit0/head0/headn   host out, [n_ctas_max]: unit a CTA starts in, its first reserved
- *                   tile there, and how many tiles it has reserved (0 or 4)
+ *                   tile there, and how many tiles it has reserved (0 or head_tiles)
  *   unit_next0      host out, [batch*kv_heads]: reserved tiles per unit = start value of the
  *                   unit's counter
  *   unit_chunk      host out, [batch*kv_heads]: tiles per pull of the unit's counter (>= 2)
  */
 mkv_status mkv_plan_starts(int batch, int kv_heads, int budget, const int32_t* prefill_lens, int n_ctas_max,
-                           int32_t* n_ctas, int32_t* cta_unit0, int32_t* cta_head0, int32_t* cta_headn,
-                           int32_t* unit_next0, int32_t* unit_chunk);
+                           int head_tiles, int32_t* n_ctas, int32_t* cta_unit0, int32_t* cta_head0,
+                           int32_t* cta_headn, int32_t* unit_next0, int32_t* unit_chunk);
+
+/*
+ * The table of the reproducible mode (MKV_FLAG_REPRODUCIBLE), as pure host arithmetic: the
+ * units' tiles (a full decode pool assumed) form one global sequence, which is cut into n_ctas
+ * contiguous ranges of near-equal length; CTA c covers tiles [cta_t0[c], cta_t0[c+1]) and its
+ * partial result for a unit goes to slot c - unit_cta0[unit].
+ *   cta_t0      host out, [n_ctas_max + 1];  tile_begin  host out, [batch*kv_heads + 1]
+ *   unit_cta0   host out, [batch*kv_heads]: first CTA whose range reaches into the unit
+ */
+mkv_status mkv_plan_ranges(int batch, int kv_heads, int budget, const int32_t* prefill_lens, int n_ctas_max,
+                           int32_t* n_ctas, int32_t* cta_t0, int32_t* tile_begin, int32_t* unit_cta0);
+
+/*
+ * Upper bound of a launch's grid: sm_count x min(resident_per_sm, wanted_per_sm), at most 2048;
+ * 0 when the kernel does not fit an SM at all (resident_per_sm < 1).  resident_per_sm is what
+ * the CUDA occupancy query reports for the kernel with its shared memory; wanted_per_sm is the
+ * design point (2 for the tensor-core kernel, 8 for the scalar one).  Pure host arithmetic;
+ * mkv_create() and MKV_OPT_RING_STAGES use it and fail with MKV_ERR_UNSUPPORTED on 0.
+ */
+int mkv_grid_limit(int sm_count, int resident_per_sm, int wanted_per_sm);
 
 /* K+V bytes one cached token occupies over all layers (the paper's 128 KB/token). */
 size_t mkv_kv_bytes_per_token(int layers, int kv_heads, int head_dim, int kv_dtype);
@@ -125,7 +189,7 @@ size_t mkv_kv_bytes_per_token(int layers, int kv_heads, int head_dim, int kv_dty
  * Create a context (Algorithm 1 "Require": decoding budget B_d = `budget`, momentum
  * factor alpha = `beta`).
  *   layers, batch            >= 1
- *   q_heads % kv_heads == 0; G = q_heads / kv_heads <= 16
+ *   q_heads % kv_heads == 0; G = q_heads / kv_heads <= 8
  *   head_dim                 64 or 128
  *   budget                   >= 1; also the largest budget mkv_set_budget accepts
  *   beta                     in [0, 1]  (paper: (0,1); 0 and 1 are the limits)
@@ -137,7 +201,8 @@ size_t mkv_kv_bytes_per_token(int layers, int kv_heads, int head_dim, int kv_dty
  *                            its first use zero-fills it on `device`'s legacy stream
  *   device                   CUDA device ordinal
  *   out_ctx                  host pointer receiving the context
- * Errors: INVALID_ARG, UNSUPPORTED (kernel family cannot do this shape), WORKSPACE, CUDA.
+ * Errors: INVALID_ARG, UNSUPPORTED (kernel family cannot do this shape, or its CTAs do not
+ * fit the device), WORKSPACE, CUDA.
  */
 mkv_status mkv_create(int layers, int q_heads, int kv_heads, int head_dim, int budget, float beta,
                       int batch, int max_prefill, int kv_dtype, int out_dtype, int score_mode,
@@ -146,6 +211,13 @@ mkv_status mkv_create(int layers, int q_heads, int kv_heads, int head_dim, int b
 
 /* Frees host state.  The workspace stays with the caller.  NULL is ignored. */
 void mkv_destroy(mkv_ctx* ctx);
+
+/*
+ * Change one of the mkv_option settings.  Options that shape the launch plan put every layer
+ * back to "not prefilled".  Errors: INVALID_ARG (unknown option, value out of range),
+ * UNSUPPORTED (option of the other kernel family; ring that does not fit), CUDA.
+ */
+mkv_status mkv_set_option(mkv_ctx* ctx, int option, long long value);
 
 /*
  * Prefill phase (Sec. 4.1): store the prompt's K_P, V_P of one layer in the frozen
@@ -185,6 +257,24 @@ mkv_status mkv_decode_step(mkv_ctx* ctx, int layer, const void* q, const void* k
                            const void* v_new, void* out, void* stream);
 
 /*
+ * The same step for layers [layer0, layer0 + n_layers) with ONE kernel launch: Algorithm 1 runs
+ * per layer and the layers' inputs are independent, so their (sequence, KV head) units simply
+ * share the grid.  Meant for small per-layer batches, where one layer alone cannot fill the GPU.
+ *   q, out            device pointers, [n_layers][batch][q_heads][head_dim]
+ *   k_new, v_new      device pointers, [n_layers][batch][kv_heads][head_dim]
+ * Every layer of the range must have been prefilled.  The first call for a range (and the first
+ * after one of its layers was prefilled again) builds the range's launch plan with copies on
+ * `stream`: make it outside stream capture.  Calls for single layers and for ranges may be
+ * mixed freely.  Errors: INVALID_ARG, BAD_STATE, CUDA.
+ */
+mkv_status mkv_decode_step_layers(mkv_ctx* ctx, int layer0, int n_layers, const void* q, const void* k_new,
+                                  const void* v_new, void* out, void* stream);
+
+/* mkv_attend_only for a run of layers with one launch; q and out as in mkv_decode_step_layers. */
+mkv_status mkv_attend_only_layers(mkv_ctx* ctx, int layer0, int n_layers, const void* q, void* out,
+                                  void* stream);
+
+/*
  * Same step with HOST buffers: copies q, k_new, v_new to the device, runs the step,
  * copies `out` back; all on `stream`, asynchronous when the host buffers are pinned
  * (the caller synchronises the stream before reading `out` or reusing the inputs).  When
@@ -192,7 +282,9 @@ mkv_status mkv_decode_step(mkv_ctx* ctx, int layer, const void* q, const void* k
  * 16-byte aligned host buffers are reached by the GPU in place: the inputs are fetched by a
  * small kernel ahead of the step and `out` is written by the step's kernel itself, instead
  * of copy operations before and after it; pageable buffers take staged copies.  Either way
- * `out` is complete once the stream has been synchronised.
+ * `out` is complete once the stream has been synchronised.  Whether a host buffer is pinned is
+ * looked up once per (address, size) and remembered until mkv_reset() or mkv_destroy(): do not
+ * unpin a buffer and hand the same address to the same context again as pageable memory.
  */
 mkv_status mkv_decode_step_host(mkv_ctx* ctx, int layer, const void* q_host, const void* k_new_host,
                                 const void* v_new_host, void* out_host, void* stream);
@@ -210,7 +302,8 @@ mkv_status mkv_attend_only(mkv_ctx* ctx, int layer, const void* q, void* out, vo
  */
 mkv_status mkv_set_budget(mkv_ctx* ctx, int budget);
 
-/* Back to "no layer prefilled"; pools keep their bytes but are treated as empty. */
+/* Back to "no layer prefilled"; pools keep their bytes but are treated as empty.  Waits for the
+ * device, then clears the sticky device status. */
 mkv_status mkv_reset(mkv_ctx* ctx);
 
 /* Synchronise `stream`, then return the sticky device status (MKV_OK if clean). */
@@ -250,6 +343,19 @@ mkv_status mkv_attend_noalloc(const void* q, const void* K, const void* V, void*
 
 /* Number of kernels this context has launched so far (host counter). */
 int64_t mkv_launch_count(const mkv_ctx* ctx);
+
+/* The grid of `layer`'s launches (0 before its prefill) and the bound it was sized under. */
+mkv_status mkv_get_grid(const mkv_ctx* ctx, int layer, int32_t* n_ctas, int32_t* n_ctas_max);
+
+/*
+ * Test hook for the error path of the bounded waits: one tile of unit (b, kv_head) of `layer`
+ * counts as never delivered from now on, so the unit's finishing part, in the next step of that
+ * layer, waits until the wait limit, gives up and sets MKV_ERR_TIMEOUT (nothing traps, nothing
+ * spins without bound; the rest of the step completes).  The layer's results are undefined
+ * afterwards: call mkv_reset() and prefill again.  Tensor-core kernel only (the scalar kernel
+ * has no waits): otherwise MKV_ERR_UNSUPPORTED.  Synchronises the device.
+ */
+mkv_status mkv_debug_withhold_tile(mkv_ctx* ctx, int layer, int b, int kv_head);
 
 /*
  * Recency-window attention diagnostics of the last decode step of `layer` (the analysis of

@@ -10,6 +10,10 @@
 //   score   [units][cap] f32             importance I_i (Eq. 5)
 //   pos     [units][cap] i32             decode-step id at which the token was appended
 //   n_dec   [units] i32                  tokens currently in the decode pool
+// Every one of these arrays is stored for all layers back to back ([layers][units]...), so a
+// run of consecutive layers is simply a longer list of units: one launch can step several
+// layers at once (Algorithm 1 runs per layer and the layers' inputs are independent), with
+// "sequence" index = layer * batch + sequence and unit index = layer * units + unit.
 //
 // A cache row is ROWB = head_dim * sizeof(element) bytes.  Rows are stored with their
 // 16-byte chunks permuted: chunk c of the row in slot s sits at chunk position
@@ -47,7 +51,9 @@ constexpr int kTileRows = 64;       // rows of one tile of the work decompositio
 constexpr int kMaxGroup = 8;        // G = q_heads / kv_heads the kernels are built for
 constexpr int kMaxParts = 64;       // partials per unit (chunks grow to keep this)
 constexpr int kMaxCtas = 2048;      // persistent grid upper bound
-constexpr int kHeadTiles = 4;       // tiles a CTA owns outright at its starting place (the ring holds 3 before the wait)
+constexpr int kHeadTiles = 4;       // tiles a CTA owns outright at its starting place, by default
+constexpr int kMaxHeadTiles = 16;   // ... and the most a context may ask for
+constexpr int kHopWindow = 256;     // units a CTA looks at, ahead of its own, when its unit runs dry
 constexpr int kMaxHome = 32;        // CTAs that start in one unit (bound kept by the start table)
 constexpr float kNegBig = -1.0e30f; // finite stand-in for -inf in running maxima
 
@@ -91,6 +97,12 @@ struct LayerDev {
     unsigned long long* keys;   // [units][cap] selection scratch
     int32_t* list_a;   // [units][cap] compaction scratch (holes)
     int32_t* list_b;   // [units][cap] compaction scratch (movers)
+    // Reproducible mode (static partition instead of counters): the global tile sequence is cut
+    // into one contiguous range per CTA.
+    const int32_t* tile_begin;  // [units + 1] first global tile of a unit (full decode pool assumed)
+    const int32_t* cta_t0;      // [n_ctas + 1] first global tile of a CTA's range
+    const int32_t* unit_cta0;   // [units] first CTA whose range reaches into the unit
+    float* unit_sum;            // [units][lstride] layer-wide score mode, reproducible: a unit's own head sums
 };
 
 struct Params {
@@ -109,6 +121,10 @@ struct Params {
     int out_f32;
     int layer_mean;    // Eq. 4 over all heads of the layer: one score vector per sequence, shared eviction
     int launch_parity; // launches of the context so far, modulo 2 (diagnostic builds keep two trace sets)
+    int early_inputs;  // the caller's q, k_new, v_new are final when the launch is enqueued: attention over
+                       // reserved prompt tiles may run before the previous kernel of the stream has completed
+    int det;           // reproducible mode: static partition, partial slots in CTA order
+    unsigned long long wait_ns;   // limit of every bounded wait inside a kernel
 };
 
 // Parity of the launch this CTA is part of; counts the launch in the CTA's own word.  Call once

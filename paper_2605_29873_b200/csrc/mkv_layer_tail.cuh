@@ -57,7 +57,23 @@ __device__ void layer_finish(const Params& p, int u, const TailPre<NT, GB>& pre,
 
     // ---- all heads: head mean, momentum update -----------------------------------------------
     const float inv_h = 1.0f / (float)Hq;
-    const float ab_new = __ldcg(sums + n_old) * inv_h;     // Eq. 6: I_fresh = alpha * 0 + abar_fresh
+    // (reproducible mode: every unit kept its own row of sums; they are added in KV-head order)
+    const float* const usums = L.unit_sum + (size_t)u0 * ls;
+    auto load_sums = [&](int i, float (&dst)[TW]) {
+        if (!p.det) { load_vec<TW>(sums + i, dst); return; }
+#pragma unroll
+        for (int j = 0; j < TW; ++j) dst[j] = 0.f;
+        for (int g2 = 0; g2 < Hkv; ++g2) {
+            float part[TW];
+            load_vec<TW>(usums + (size_t)g2 * ls + i, part);
+#pragma unroll
+            for (int j = 0; j < TW; ++j) dst[j] += part[j];
+        }
+    };
+    float sum_fresh = 0.f;
+    if (p.det) { for (int g2 = 0; g2 < Hkv; ++g2) sum_fresh += __ldcg(usums + (size_t)g2 * ls + n_old); }
+    else sum_fresh = __ldcg(sums + n_old);
+    const float ab_new = sum_fresh * inv_h;                // Eq. 6: I_fresh = alpha * 0 + abar_fresh
     const unsigned long long key_new = ((unsigned long long)__float_as_uint(ab_new) << 32) | (unsigned)t;
     unsigned long long* keys = L.keys + (size_t)u0 * cap;
     const float* score0 = L.score + (size_t)u0 * ls;
@@ -107,8 +123,8 @@ __device__ void layer_finish(const Params& p, int u, const TailPre<NT, GB>& pre,
         const int ia = base + TW * tid, ib = ia + TW * NT;
         float sa[TW], sca[TW], sb[TW], scb[TW];
         int psa[TW], psb[TW];
-        if (ia < n_old) { load_vec<TW>(sums + ia, sa); load_vec<TW>(score0 + ia, sca); load_vec<TW>(pos0 + ia, psa); }
-        if (ib < n_old) { load_vec<TW>(sums + ib, sb); load_vec<TW>(score0 + ib, scb); load_vec<TW>(pos0 + ib, psb); }
+        if (ia < n_old) { load_sums(ia, sa); load_vec<TW>(score0 + ia, sca); load_vec<TW>(pos0 + ia, psa); }
+        if (ib < n_old) { load_sums(ib, sb); load_vec<TW>(score0 + ib, scb); load_vec<TW>(pos0 + ib, psb); }
         token_pass(ia, sa, sca, psa);
         token_pass(ib, sb, scb, psb);
     }

@@ -32,10 +32,19 @@
 //   * four TAIL warps, which watch the counts of the units assigned to this CTA and run a
 //     unit's tail (fresh token, combine, probabilities, momentum update, selection,
 //     append/compaction) as soon as its count is complete, while the stream continues.
-// Every wait is bounded: on expiry the kernel records MKV_ERR_TIMEOUT, every role drains
-// (the producer waits, bounded again, for its copies in flight) and the CTA returns.
-#include <cstdlib>
-
+// Every wait is bounded (the context's wait limit): on expiry the kernel records
+// MKV_ERR_TIMEOUT, every role drains (the producer waits, bounded again, for its copies in
+// flight) and the CTA returns.
+//
+// CTAs wait on one another (a unit's tail waits for tiles other CTAs deliver), so the whole
+// grid has to be resident at once: the host sizes it from the occupancy the device reports.
+//
+// Two optional behaviours, both decided by the context:
+//   * early inputs: the caller's q is final when the launch is enqueued, so the consumers may
+//     work through the CTA's reserved prompt tiles (frozen rows) while the previous kernel of
+//     the stream is still running its last tails; everything else waits for it as usual.
+//   * reproducible mode: no counters; every CTA covers a fixed range of the global tile
+//     sequence and delivers a fixed partial slot, so the same inputs give the same bits.
 #include "mkv_launch.h"
 #include "mkv_ptx.cuh"
 #include "mkv_layer_tail.cuh"
@@ -59,7 +68,7 @@ constexpr int kTailTid0 = (kMergeWarp + 1) * 32;          // first thread of the
 constexpr int kThreads = kTailTid0 + kTailThreads;
 constexpr int kMaxStages = 8;
 constexpr int kXoStride = 132;                            // floats per head row of the exchange
-constexpr unsigned long long kWaitNs = 2000000000ull;     // 2 s
+constexpr size_t kSmemPerCta = 232448;                    // opt-in shared memory of one CTA on sm_100
 
 enum : int { kEntryTile = 0, kEntryExchange = 1, kEntryEnd = 2 };
 
@@ -73,7 +82,7 @@ struct StageMeta {
     int slot;       // exchange entries: the visit's partial slot ...
     int ntiles;     // ... the tiles it covered ...
     int total;      // ... and the unit's tile count
-    int pad;
+    int pre;        // issued before the dependency wait: touches nothing an earlier kernel writes
 };
 
 struct ExchangeRef { int stage, unit, slot, ntiles, total; };   // stage < 0: no more exchanges
@@ -103,7 +112,7 @@ __device__ inline void note_timeout(const Params& p, Control* ctl) {
 }
 
 // Bounded mbarrier wait that also gives up as soon as another role has aborted.
-__device__ inline bool wait_or_abort(uint32_t bar, uint32_t parity, Control* ctl) {
+__device__ inline bool wait_or_abort(uint32_t bar, uint32_t parity, Control* ctl, unsigned long long limit_ns) {
     for (int i = 0; i < 32; ++i)
         if (ptx::mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = ptx::globaltimer_ns();
@@ -111,7 +120,7 @@ __device__ inline bool wait_or_abort(uint32_t bar, uint32_t parity, Control* ctl
         for (int i = 0; i < 128; ++i)
             if (ptx::mbar_try_wait(bar, parity)) return true;
         if (aborted(ctl)) return false;
-        if (ptx::globaltimer_ns() - t0 > kWaitNs) return false;
+        if (ptx::globaltimer_ns() - t0 > limit_ns) return false;
     }
 }
 
@@ -128,7 +137,8 @@ __device__ void tail_group(const Params& p, Control* ctl, TailSmem<kTailThreads>
         TailPre<kTailThreads, GB> pre;
         tail_prefetch<__nv_bfloat16, kTailThreads, GB, LAYER>(p, u, *tsm, tt, pre);
         if (tt == 0) {
-            const int total = unit_tiles(L.unit_lp[u], min(pre.n_dec, p.cap - (dec ? 1 : 0)));
+            const int total = p.det ? L.tile_begin[u + 1] - L.tile_begin[u]
+                                    : unit_tiles(L.unit_lp[u], min(pre.n_dec, p.cap - (dec ? 1 : 0)));
             const unsigned long long t0 = ptx::globaltimer_ns();
             int slots = -1;
             int par = tsm->par;
@@ -136,14 +146,14 @@ __device__ void tail_group(const Params& p, Control* ctl, TailSmem<kTailThreads>
                 par = *reinterpret_cast<const volatile int*>(&ctl->par);
                 if (par >= 0) { tsm->par = par; break; }
                 if (aborted(ctl)) break;
-                if (ptx::globaltimer_ns() - t0 > kWaitNs) { note_timeout(p, ctl); break; }
+                if (ptx::globaltimer_ns() - t0 > p.wait_ns) { note_timeout(p, ctl); break; }
             }
             const int2* cnt_u = L.cnt + (size_t)max(par, 0) * L.n_units + u;
             for (; par >= 0;) {
                 const unsigned long long w = *reinterpret_cast<const volatile unsigned long long*>(cnt_u);
                 if ((int)(unsigned)(w & 0xffffffffull) >= total) { slots = (int)(unsigned)(w >> 32); break; }
                 if (aborted(ctl)) break;
-                if (ptx::globaltimer_ns() - t0 > kWaitNs) { note_timeout(p, ctl); break; }
+                if (ptx::globaltimer_ns() - t0 > p.wait_ns) { note_timeout(p, ctl); break; }
                 __nanosleep(100);
             }
             ctl->tail_unit = slots;
@@ -209,7 +219,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         const unsigned long long stream_policy = ptx::l2_policy_evict_first();
         int qcount = 0;            // visits that had at least one tile (and therefore a query slot)
         auto acquire = [&]() -> bool {
-            if (!wait_or_abort(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl)) {
+            if (!wait_or_abort(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, p.wait_ns)) {
                 if (!aborted(ctl)) note_timeout(p, ctl);
                 return false;
             }
@@ -217,10 +227,11 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             return true;
         };
         auto advance = [&]() { if (++stage == nst) { stage = 0; phase ^= 1u; } };
-        auto issue_tile = [&](int u, const TileRef& tr, int first) -> bool {
+        auto issue_tile = [&](int u, const TileRef& tr, int first, int pre) -> bool {
             if (!acquire()) return false;
             StageMeta& mt = ctl->meta[stage];
             mt.kind = kEntryTile; mt.unit = u; mt.seg = tr.seg; mt.row = tr.row; mt.cnt = tr.cnt; mt.first = first;
+            mt.pre = pre;
             const uint32_t fb = ptx::smem_u32(&ctl->full[stage]);
             const uint32_t dstK = ptx::smem_u32(stages + (size_t)stage * kStageBytes);
             const size_t off = ((size_t)u * (tr.seg == 0 ? p.max_prefill : p.cap) + tr.row) * kRowB;
@@ -239,7 +250,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         auto issue_query = [&](int u) -> bool {
             const int b = u / p.kv_heads, g = u - b * p.kv_heads;
             const int qi = qcount & 1;
-            if (!wait_or_abort(ptx::smem_u32(&ctl->qempty[qi]), (uint32_t)(((qcount >> 1) & 1) ^ 1), ctl)) {
+            if (!wait_or_abort(ptx::smem_u32(&ctl->qempty[qi]), (uint32_t)(((qcount >> 1) & 1) ^ 1), ctl, p.wait_ns)) {
                 if (!aborted(ctl)) note_timeout(p, ctl);
                 return false;
             }
@@ -270,12 +281,17 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         // touched: the start table and the frozen prefill pool.  The CTA's reserved tiles (prefill
         // tiles by construction) are therefore in flight while the previous step still runs.
         int head_t = 0, head_end = 0;   // reserved tiles still to issue (lane 0)
+        const bool early = p.early_inputs != 0;
         if (lane == 0) {
             head_t = L.cta_head0[blockIdx.x];
             head_end = head_t + L.cta_headn[blockIdx.x];
-            // no more than the ring holds: the consumers only start after the wait
-            for (int n = 0; head_t < head_end && n < nst && ok; ++n, ++head_t) {
-                ok = issue_tile(u, tile_ref(head_t, lp, 0), sent == 0);
+            // With early inputs the query is final already and the consumers work through the
+            // reserved tiles now; otherwise no more than the ring holds, for the consumers only
+            // start after the wait.
+            if (early && head_t < head_end) { ok = issue_query(u); q_sent = true; }
+            const int before = early ? head_end - head_t : nst;
+            for (int n = 0; head_t < head_end && n < before && ok; ++n, ++head_t) {
+                ok = issue_tile(u, tile_ref(head_t, lp, 0), sent == 0, early ? 1 : 0);
                 if (ok) { if (sent == 0) MKV_TR(1); ++sent; ++mine; }
             }
         }
@@ -287,7 +303,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         uint32_t seen = 0;         // launches this CTA has taken part in (lane 0)
         if (lane == 0) seen = __ldcg(&L.launch_no[blockIdx.x]);
         const bool has_head = head_end > L.cta_head0[blockIdx.x];
-        if (lane == 0 && ok && has_head) {
+        if (lane == 0 && ok && has_head && !q_sent) {
             ok = issue_query(u);
             q_sent = true;
         }
@@ -307,13 +323,42 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         if (lane == 0 && ok && has_head) {
             slot = atomicAdd(&cnt[u].y, 1);
             for (; head_t < head_end && ok; ++head_t) {
-                ok = issue_tile(u, tile_ref(head_t, lp, 0), sent == 0);
+                ok = issue_tile(u, tile_ref(head_t, lp, 0), sent == 0, 0);
                 ++sent; ++mine;
             }
         }
+        // Reproducible mode: this CTA's fixed range of the global tile sequence, unit by unit; the
+        // partial of a unit visit goes to the slot that is this CTA's rank among the unit's CTAs.
+        if (p.det && lane == 0 && ok) {
+            int t = L.cta_t0[blockIdx.x];
+            const int t_end = L.cta_t0[blockIdx.x + 1];
+            for (int uu = u; t < t_end && ok; ++uu) {
+                const int ub = L.tile_begin[uu], ue = L.tile_begin[uu + 1];
+                const int lpu = L.unit_lp[uu];
+                const int ndu = min(L.n_dec[uu], p.cap - (dec ? 1 : 0));
+                const int a = t - ub, b = min(t_end, ue) - ub;
+                atomicAdd(&cnt[uu].y, 1);                      // visits of the unit (the tail's partial count)
+                int sent_u = 0;
+                for (int tt = a; tt < b && ok; ++tt) {
+                    const TileRef tr = tile_ref(tt, lpu, ndu);
+                    if (tr.cnt == 0) continue;
+                    if (sent_u == 0 && !(ok = issue_query(uu))) break;
+                    ok = issue_tile(uu, tr, sent_u == 0, 0);
+                    ++sent_u;
+                }
+                if (ok && (ok = acquire())) {
+                    StageMeta& mt = ctl->meta[stage];
+                    mt.kind = kEntryExchange; mt.unit = uu; mt.seg = 0; mt.row = 0; mt.cnt = 0; mt.first = (sent_u == 0);
+                    mt.slot = (int)blockIdx.x - L.unit_cta0[uu]; mt.ntiles = b - a; mt.total = ue - ub; mt.pre = 0;
+                    ptx::mbar_arrive(ptx::smem_u32(&ctl->full[stage]));
+                    advance();
+                }
+                t = ub + b;
+            }
+        }
         int g = 0;                 // first tile of the chunk in hand
-        if (lane == 0) g = atomicAdd(&nxt[u], chunk);
-        for (;;) {
+        if (lane == 0 && !p.det) g = atomicAdd(&nxt[u], chunk);
+        for (; !p.det;) {
             g = __shfl_sync(0xffffffffu, g, 0);
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
@@ -327,7 +372,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
                         ++mine;
                         if (tr.cnt == 0) continue;
                         if (!q_sent) { ok = issue_query(u); q_sent = true; if (!ok) break; }
-                        ok = issue_tile(u, tr, sent == 0);
+                        ok = issue_tile(u, tr, sent == 0, 0);
                         ++sent;
                     }
                     g = g_next;
@@ -339,7 +384,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
                 if ((ok = acquire())) {
                     StageMeta& mt = ctl->meta[stage];
                     mt.kind = kEntryExchange; mt.unit = u; mt.seg = 0; mt.row = 0; mt.cnt = 0; mt.first = (sent == 0);
-                    mt.slot = slot; mt.ntiles = mine; mt.total = total;
+                    mt.slot = slot; mt.ntiles = mine; mt.total = total; mt.pre = 0;
                     ptx::mbar_arrive(ptx::smem_u32(&ctl->full[stage]));
                     advance();
                 }
@@ -349,7 +394,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             if (!ok) break;
             // ... and look for the next unit (cyclically after this one) that still has some.
             int found = -1;
-            for (int base = 1; base < U && found < 0; base += 32) {
+            for (int base = 1; base < U && base <= kHopWindow && found < 0; base += 32) {
                 const int k = base + lane;
                 int lpc = 0, ndc = 0, rem = 0, chc = 2;
                 if (k < U) {
@@ -380,19 +425,22 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         if (lane == 0) {
             if (ok && acquire()) {
                 ctl->meta[stage].kind = kEntryEnd;
+                ctl->meta[stage].pre = 0;
                 ptx::mbar_arrive(ptx::smem_u32(&ctl->full[stage]));
             } else {
                 // abort: leave only after every copy this thread issued has landed
                 for (int s2 = 0; s2 < nst; ++s2)
                     if (issued & (1u << s2))
-                        wait_or_abort(ptx::smem_u32(&ctl->full[s2]), (issued_par >> s2) & 1u, ctl) ||
-                            ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->full[s2]), (issued_par >> s2) & 1u, kWaitNs);
+                        ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->full[s2]), (issued_par >> s2) & 1u, p.wait_ns);
             }
         }
         __syncwarp();
     } else if (warp < kConsumerWarps) {
         // ================================ consumers ====================================
-        ptx::griddep_wait();
+        // They pass the dependency wait at the first entry that was issued after the producer's
+        // own: entries issued before it (reserved prompt tiles, with early inputs) read frozen
+        // rows and the caller's query only, and change nothing but registers.
+        bool waited = false;
         int stage = 0;
         uint32_t phase = 0;
         int xcount = 0;
@@ -408,11 +456,12 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         for (int j = 0; j < 8; ++j) { oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f; }
 
         for (;;) {
-            if (!wait_or_abort(ptx::smem_u32(&ctl->full[stage]), phase, ctl)) {
+            if (!wait_or_abort(ptx::smem_u32(&ctl->full[stage]), phase, ctl, p.wait_ns)) {
                 if (lane == 0 && !aborted(ctl)) note_timeout(p, ctl);
                 break;
             }
             const StageMeta mt = ctl->meta[stage];
+            if (!waited && !mt.pre) { ptx::griddep_wait(); waited = true; }
             if (warp == 0 && lane == 0 && xcount == 0 && mt.first) MKV_TR(2);
             if (mt.kind == kEntryEnd) {
                 if (warp == 0 && lane == 0) MKV_TR(3);
@@ -434,7 +483,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
                 }
                 if (mt.kind == kEntryTile) {
                     const int qi = qcount & 1;
-                    if (!wait_or_abort(ptx::smem_u32(&ctl->qfull[qi]), (uint32_t)((qcount >> 1) & 1), ctl)) {
+                    if (!wait_or_abort(ptx::smem_u32(&ctl->qfull[qi]), (uint32_t)((qcount >> 1) & 1), ctl, p.wait_ns)) {
                         if (lane == 0 && !aborted(ctl)) note_timeout(p, ctl);
                         break;
                     }
@@ -557,7 +606,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         ptx::griddep_wait();
         for (int x = 0;; ++x) {
             const int xs = x % nst;
-            if (!wait_or_abort(ptx::smem_u32(&ctl->xfull[xs]), (uint32_t)((x / nst) & 1), ctl)) {
+            if (!wait_or_abort(ptx::smem_u32(&ctl->xfull[xs]), (uint32_t)((x / nst) & 1), ctl, p.wait_ns)) {
                 if (lane == 0 && !aborted(ctl)) note_timeout(p, ctl);
                 break;
             }
@@ -619,8 +668,6 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
     }
 }
 
-int g_stages = 3;
-
 }  // namespace
 
 #ifdef MKV_TRACE
@@ -633,22 +680,43 @@ bool mma_supported(int kv_dtype, int head_dim, int group) {
     return kv_dtype == 0 && head_dim == 128 && group >= 1 && group <= kMaxGroup;
 }
 
-cudaError_t mma_configure() {
-    if (const char* e = std::getenv("MKV_STAGES")) g_stages = max(2, min(kMaxStages, atoi(e)));
-    cudaError_t e = cudaFuncSetAttribute(mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(g_stages));
+int mma_max_stages() {
+    int n = 2;
+    while (n < kMaxStages && smem_bytes(n + 1) <= kSmemPerCta) ++n;
+    return n;
+}
+
+// CTAs of the kernel an SM keeps resident with a ring of `stages` stages.  Also raises the
+// kernels' dynamic shared memory limit to what that ring needs.
+cudaError_t mma_occupancy(int stages, int* resident_per_sm) {
+    static size_t opted = 0;       // the limit is a per-function maximum: it only ever grows
+    const size_t need = smem_bytes(stages);
+    if (need > kSmemPerCta) return cudaErrorInvalidValue;
+    if (need > opted) {
+        cudaError_t e = cudaFuncSetAttribute(mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+        if (e != cudaSuccess) return e;
+        opted = need;
+    }
+    int a = 0, b = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, mma_kernel<false>, kThreads, need);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes(g_stages));
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, mma_kernel<true>, kThreads, need);
+    if (e != cudaSuccess) return e;
+    *resident_per_sm = a < b ? a : b;
+    return cudaSuccess;
 }
 
 // overlap: launch with programmatic stream serialization, i.e. this kernel's CTAs may start
 // while the previous kernel of the stream is still finishing; the kernel itself waits
 // (griddepcontrol.wait) before it touches anything an earlier kernel may write.
-cudaError_t launch_mma(const Params& p, cudaStream_t st, bool overlap) {
+cudaError_t launch_mma(const Params& p, cudaStream_t st, bool overlap, int stages) {
     if (p.L.n_ctas <= 0) return cudaSuccess;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.L.n_ctas);
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem_bytes(g_stages);
+    cfg.dynamicSmemBytes = smem_bytes(stages);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -656,8 +724,8 @@ cudaError_t launch_mma(const Params& p, cudaStream_t st, bool overlap) {
     cfg.attrs = attr;
     cfg.numAttrs = overlap ? 1 : 0;
     // the layer-wide score mode has its own instantiation, so that neither carries the other's tail
-    if (p.layer_mean) return cudaLaunchKernelEx(&cfg, mma_kernel<true>, p, g_stages);
-    return cudaLaunchKernelEx(&cfg, mma_kernel<false>, p, g_stages);
+    if (p.layer_mean) return cudaLaunchKernelEx(&cfg, mma_kernel<true>, p, stages);
+    return cudaLaunchKernelEx(&cfg, mma_kernel<false>, p, stages);
 }
 
 }  // namespace mkv

@@ -9,7 +9,9 @@
 // row (GQA).  Per row: G dot products (Eq. 2 logits, already in log2 units), a butterfly
 // warp reduction, an online-softmax update of (m, l, O).  At the end of a unit visit the warps
 // are merged in shared memory and the CTA writes one partial with its tile count; the
-// delivery that completes the unit runs its tail.
+// delivery that completes the unit runs its tail.  In the reproducible mode there are no
+// counters: every CTA covers a fixed range of the global tile sequence and its partial of a
+// unit goes to a fixed slot.
 #include "mkv_launch.h"
 #include "mkv_layer_tail.cuh"
 #include "mkv_tail.cuh"
@@ -65,7 +67,11 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
 
     int u = L.cta_unit0[blockIdx.x];
     int head = L.cta_head0[blockIdx.x], headn = L.cta_headn[blockIdx.x];   // reserved tiles, first visit only
+    const bool det = p.det != 0;
+    int det_t = det ? L.cta_t0[blockIdx.x] : 0;                 // reproducible mode: next global tile ...
+    const int det_end = det ? L.cta_t0[blockIdx.x + 1] : 0;     // ... and the end of this CTA's range
     for (;;) {
+        if (det && det_t >= det_end) break;
         // ---- one visit of unit u: pull chunks until the unit has none left -------------------
         const int b = u / p.kv_heads, g = u - b * p.kv_heads;
         const int lp = L.unit_lp[u];
@@ -74,7 +80,9 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
             if (tid == 0) atomicCAS(p.status, kStatusOk, kStatusDeviceCheck);
             n_old = p.cap - (dec ? 1 : 0);
         }
-        const int total = unit_tiles(lp, n_old), chunk = L.unit_chunk[u];
+        const int chunk = L.unit_chunk[u];
+        const int total = det ? L.tile_begin[u + 1] - L.tile_begin[u] : unit_tiles(lp, n_old);
+        bool det_taken = false;
         float qf[G][EPL];
         {
             const T* qp = reinterpret_cast<const T*>(p.q) + ((size_t)b * p.q_heads + (size_t)g * G) * D + lane * EPL;
@@ -94,7 +102,13 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
         int mine = 0;
         for (;;) {
             int t0, t1;
-            if (headn > 0) { t0 = head; t1 = head + headn; headn = 0; }
+            if (det) {
+                if (det_taken) break;
+                det_taken = true;
+                t0 = det_t - L.tile_begin[u];
+                t1 = min(det_end, L.tile_begin[u + 1]) - L.tile_begin[u];
+                det_t = L.tile_begin[u] + t1;
+            } else if (headn > 0) { t0 = head; t1 = head + headn; headn = 0; }
             else {
                 if (tid == 0) s_g = atomicAdd(&nxt[u], chunk);
                 __syncthreads();
@@ -142,7 +156,10 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
         }
         if (mine > 0) {
             // merge the four warps, write the visit's partial into a fresh slot of the unit
-            if (tid == 0) s_g = atomicAdd(&cnt[u].y, 1);
+            if (tid == 0) {
+                s_g = atomicAdd(&cnt[u].y, 1);
+                if (det) s_g = (int)blockIdx.x - L.unit_cta0[u];    // a fixed slot: this CTA's rank in the unit
+            }
             if (lane == 0) {
 #pragma unroll
                 for (int h = 0; h < G; ++h) { xm[warp][h] = m[h]; xl[warp][h] = l[h]; }
@@ -192,9 +209,10 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
             __syncthreads();
         }
         // ---- next unit (cyclically after this one) that still has tiles to hand out -----------
+        if (det) { ++u; if (u >= U) break; continue; }
         if (tid == 0) {
             int found = -1;
-            for (int k = 1; k < U; ++k) {
+            for (int k = 1; k < U && k <= kHopWindow; ++k) {
                 const int cand = (u + k) % U;
                 const int nd = min(L.n_dec[cand], p.cap - (dec ? 1 : 0));
                 if (__ldcg(&nxt[cand]) < unit_tiles(L.unit_lp[cand], nd)) { found = cand; break; }
@@ -220,7 +238,25 @@ cudaError_t launch_td(const Params& p, cudaStream_t st) {
     return cudaGetLastError();
 }
 
+template <typename T, int D>
+cudaError_t occupancy_td(int group, int* n) {
+    switch (group) {
+#define MKV_CASE(GG) case GG: return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, simt_kernel<T, D, GG>, kSimtThreads, 0);
+        MKV_CASE(1) MKV_CASE(2) MKV_CASE(3) MKV_CASE(4) MKV_CASE(5) MKV_CASE(6) MKV_CASE(7) MKV_CASE(8)
+#undef MKV_CASE
+        default: return cudaErrorInvalidValue;
+    }
+}
+
 }  // namespace
+
+cudaError_t simt_occupancy(int kv_dtype, int head_dim, int group, int* resident_per_sm) {
+    if (kv_dtype == 0)
+        return head_dim == 128 ? occupancy_td<__nv_bfloat16, 128>(group, resident_per_sm)
+                               : occupancy_td<__nv_bfloat16, 64>(group, resident_per_sm);
+    return head_dim == 128 ? occupancy_td<float, 128>(group, resident_per_sm)
+                           : occupancy_td<float, 64>(group, resident_per_sm);
+}
 
 bool simt_supported(int kv_dtype, int head_dim, int group) {
     return (kv_dtype == 0 || kv_dtype == 1) && (head_dim == 64 || head_dim == 128) && group >= 1 && group <= kMaxGroup;

@@ -189,8 +189,9 @@ __device__ void tail_prefetch(const Params& p, int u, TailSmem<NT>& sm, int tid,
 // LAYER (score mode "mean over all heads of the layer"): the tail stops after `out` and the
 // probabilities.  Per decode token it adds the SUM over the unit's G heads of the normalised
 // probabilities (the fresh token's at index n_old) to the sequence's row of head sums (vector
-// atomics); scores, selection and compaction follow for all KV heads of the sequence together
-// (layer_finish).
+// atomics; in the reproducible mode it stores them in a row of its own instead, and the rows
+// are added up in KV-head order later); scores, selection and compaction follow for all KV
+// heads of the sequence together (layer_finish).
 template <typename T, int NT, int BAR, int GB, bool LAYER = false>
 __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB>& pre, TailSmem<NT>& sm, int tid) {
     const LayerDev& L = p.L;
@@ -214,6 +215,7 @@ __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB
     int32_t* pos = L.pos + (size_t)u * ls;
     const float* lg = L.logit + ((size_t)b * p.q_heads + (size_t)g * G) * ls;
     float* psum = L.head_sum + (size_t)b * ls;                              // LAYER only
+    float* usum = L.unit_sum + (size_t)u * ls;                              // LAYER, reproducible mode
     const float* po_base = L.part_o + (size_t)part0 * G * D;
     const size_t pstride = (size_t)G * D;
     const int ne = G * D / 4;                           // float4 elements of one partial / of `out`
@@ -360,7 +362,10 @@ __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB
             }
         }
         if constexpr (LAYER) {
-            if (i0 + TW <= n_old) {
+            if (p.det) {
+#pragma unroll
+                for (int j = 0; j < TW; ++j) if (i0 + j < n_old) usum[i0 + j] = ab[j];
+            } else if (i0 + TW <= n_old) {
                 if constexpr (TW == 4) atomicAdd(reinterpret_cast<float4*>(psum + i0), make_float4(ab[0], ab[1], ab[2], ab[3]));
                 else atomicAdd(reinterpret_cast<float2*>(psum + i0), make_float2(ab[0], ab[1]));
             } else {
@@ -412,7 +417,10 @@ __device__ void unit_tail(const Params& p, int u, int P_in, const TailPre<NT, GB
     if (!out_done) finish_out();
     if (tid == 0) MKV_TR(12);
     if constexpr (LAYER) {
-        if (tid == NT - 1) atomicAdd(psum + n_old, sum_new);
+        if (tid == NT - 1) {
+            if (p.det) usum[n_old] = sum_new;
+            else atomicAdd(psum + n_old, sum_new);
+        }
         return;
     }
     if (tid == NT - 1) {                              // the fresh token sits (virtually) in slot n_old

@@ -12,7 +12,8 @@ import numpy as np
 MKV_BF16, MKV_F32 = 0, 1
 MKV_SCORE_GROUP_MEAN, MKV_SCORE_LAYER_MEAN = 0, 1
 MKV_KERNEL_AUTO, MKV_KERNEL_SIMT, MKV_KERNEL_MMA = 0, 1, 2
-MKV_FLAG_RECORD_PROBS = 1
+MKV_FLAG_RECORD_PROBS, MKV_FLAG_INPUTS_READY, MKV_FLAG_REPRODUCIBLE = 1, 2, 4
+MKV_OPT_RING_STAGES, MKV_OPT_HEAD_TILES, MKV_OPT_WAIT_LIMIT_US, MKV_OPT_OVERLAP = 1, 2, 3, 4
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmkv.so")
@@ -22,7 +23,8 @@ EXPORTED_SYMBOLS = [
     "mkv_decode_step", "mkv_decode_step_host", "mkv_attend_only", "mkv_set_budget", "mkv_reset",
     "mkv_status_sync", "mkv_launch_count", "mkv_get_decode_state", "mkv_get_last_evicted",
     "mkv_get_last_probs", "mkv_read_kv", "mkv_get_step", "mkv_status_string", "mkv_attend_noalloc", "mkv_plan_starts", "mkv_prefill_units",
-    "mkv_recency_diagnostics",
+    "mkv_recency_diagnostics", "mkv_set_option", "mkv_plan_ranges", "mkv_grid_limit", "mkv_decode_step_layers",
+    "mkv_attend_only_layers", "mkv_get_grid", "mkv_debug_withhold_tile",
 ]
 
 
@@ -70,7 +72,15 @@ def load_library(path: str | None = None):
     L.mkv_read_kv.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, i32p, vp, vp, C.c_int]
     L.mkv_get_step.argtypes = [vp, C.c_int, C.POINTER(C.c_int64)]
     L.mkv_attend_noalloc.argtypes = [vp, vp, vp, vp] + [C.c_int] * 9 + [vp]
-    L.mkv_plan_starts.argtypes = [C.c_int, C.c_int, C.c_int, i32p, C.c_int, i32p, i32p, i32p, i32p, i32p, i32p]
+    L.mkv_plan_starts.argtypes = [C.c_int, C.c_int, C.c_int, i32p, C.c_int, C.c_int, i32p, i32p, i32p, i32p, i32p, i32p]
+    L.mkv_plan_ranges.argtypes = [C.c_int, C.c_int, C.c_int, i32p, C.c_int, i32p, i32p, i32p, i32p]
+    L.mkv_grid_limit.restype = C.c_int
+    L.mkv_grid_limit.argtypes = [C.c_int, C.c_int, C.c_int]
+    L.mkv_set_option.argtypes = [vp, C.c_int, C.c_longlong]
+    L.mkv_decode_step_layers.argtypes = [vp, C.c_int, C.c_int, vp, vp, vp, vp, vp]
+    L.mkv_attend_only_layers.argtypes = [vp, C.c_int, C.c_int, vp, vp, vp]
+    L.mkv_get_grid.argtypes = [vp, C.c_int, i32p, i32p]
+    L.mkv_debug_withhold_tile.argtypes = [vp, C.c_int, C.c_int, C.c_int]
     L.mkv_status_string.restype = C.c_char_p
     L.mkv_status_string.argtypes = [C.c_int]
     if path is None:
@@ -111,7 +121,26 @@ def attend_noalloc(q, K, V, out, n_tokens, stream=None):
            "mkv_attend_noalloc")
 
 
-def plan_starts(batch, kv_heads, budget, prefill_lens, n_ctas_max):
+def grid_limit(sm_count, resident_per_sm, wanted_per_sm) -> int:
+    return int(load_library().mkv_grid_limit(sm_count, resident_per_sm, wanted_per_sm))
+
+
+def plan_ranges(batch, kv_heads, budget, prefill_lens, n_ctas_max):
+    """The table of the reproducible mode (``mkv_plan_ranges``; host arithmetic only).
+    Returns (cta_t0 [n_ctas+1], tile_begin [units+1], unit_cta0 [units]) as int32 arrays."""
+    lens = np.ascontiguousarray(prefill_lens, dtype=np.int32)
+    assert lens.shape == (batch,)
+    n = C.c_int32(0)
+    t0 = np.zeros(n_ctas_max + 1, dtype=np.int32)
+    tb = np.zeros(batch * kv_heads + 1, dtype=np.int32)
+    uc = np.zeros(batch * kv_heads, dtype=np.int32)
+    p = lambda a: a.ctypes.data_as(C.POINTER(C.c_int32))
+    _check(load_library().mkv_plan_ranges(batch, kv_heads, budget, p(lens), n_ctas_max, C.byref(n), p(t0), p(tb), p(uc)),
+           "mkv_plan_ranges")
+    return t0[: n.value + 1].copy(), tb, uc
+
+
+def plan_starts(batch, kv_heads, budget, prefill_lens, n_ctas_max, head_tiles=4):
     """The kernels' start table for these lengths (``mkv_plan_starts``; host arithmetic only).
     Returns (cta_unit0, cta_head0, cta_headn, unit_next0, unit_chunk) as int32 arrays."""
     lens = np.ascontiguousarray(prefill_lens, dtype=np.int32)
@@ -121,8 +150,8 @@ def plan_starts(batch, kv_heads, budget, prefill_lens, n_ctas_max):
     nx = np.zeros(batch * kv_heads, dtype=np.int32)
     ch = np.zeros(batch * kv_heads, dtype=np.int32)
     p = lambda a: a.ctypes.data_as(C.POINTER(C.c_int32))
-    _check(load_library().mkv_plan_starts(batch, kv_heads, budget, p(lens), n_ctas_max, C.byref(n), p(u0), p(h0), p(hn),
-                                          p(nx), p(ch)), "mkv_plan_starts")
+    _check(load_library().mkv_plan_starts(batch, kv_heads, budget, p(lens), n_ctas_max, head_tiles, C.byref(n), p(u0),
+                                          p(h0), p(hn), p(nx), p(ch)), "mkv_plan_starts")
     return u0[: n.value].copy(), h0[: n.value].copy(), hn[: n.value].copy(), nx, ch
 
 
@@ -223,6 +252,27 @@ class MomentKV:
 
     def attend_only(self, layer, q, out, stream=None):
         _check(self._L.mkv_attend_only(self._ctx, layer, _ptr(q), _ptr(out), self._stream(stream)), "mkv_attend_only")
+
+    def decode_step_layers(self, layer0, n_layers, q, k_new, v_new, out, stream=None):
+        """One launch for layers [layer0, layer0 + n_layers); tensors stacked by layer in front."""
+        _check(self._L.mkv_decode_step_layers(self._ctx, layer0, n_layers, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out),
+                                              self._stream(stream)), "mkv_decode_step_layers")
+
+    def attend_only_layers(self, layer0, n_layers, q, out, stream=None):
+        _check(self._L.mkv_attend_only_layers(self._ctx, layer0, n_layers, _ptr(q), _ptr(out), self._stream(stream)),
+               "mkv_attend_only_layers")
+
+    def set_option(self, option, value):
+        _check(self._L.mkv_set_option(self._ctx, int(option), int(value)), "mkv_set_option")
+
+    def grid(self, layer):
+        """(CTAs of the layer's launches, the bound the grid was sized under)."""
+        n, nmax = C.c_int32(0), C.c_int32(0)
+        _check(self._L.mkv_get_grid(self._ctx, layer, C.byref(n), C.byref(nmax)), "mkv_get_grid")
+        return int(n.value), int(nmax.value)
+
+    def debug_withhold_tile(self, layer, b, g):
+        _check(self._L.mkv_debug_withhold_tile(self._ctx, layer, b, g), "mkv_debug_withhold_tile")
 
     def set_budget(self, budget):
         _check(self._L.mkv_set_budget(self._ctx, int(budget)), "mkv_set_budget")

@@ -62,7 +62,9 @@ def test_workspace_bytes_rejects_bad_shapes(lib):
     assert mkv.workspace_bytes(1, 1, 4, 1, 96, 64, 64) == 0      # head_dim
     assert mkv.workspace_bytes(0, 1, 4, 1, 64, 64, 64) == 0
     assert mkv.workspace_bytes(1, 1, 4, 1, 64, 0, 64) == 0       # budget >= 1
-    assert mkv.workspace_bytes(1, 1, 64, 1, 64, 64, 64) == 0     # group > 16
+    assert mkv.workspace_bytes(1, 1, 64, 1, 64, 64, 64) == 0     # group > 8
+    assert mkv.workspace_bytes(1, 1, 9, 1, 64, 64, 64) == 0      # (the sizing call and mkv_create agree)
+    assert mkv.workspace_bytes(1, 1, 8, 1, 64, 64, 64) > 0
 
 
 def test_create_validates_then_fails_loudly_without_a_gpu(lib):
