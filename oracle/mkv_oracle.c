@@ -114,6 +114,26 @@ void mko_prefill(mko_state *s, const double *K, const double *V) {
 void mko_set_budget(mko_state *s, int budget) { if (budget >= 1) s->budget = budget; }
 
 /*
+ * State loader (no arithmetic): puts KV head g's decode pool into a given state -- n tokens
+ * with keys, values, importances and position ids, in the given order -- and sets the number of
+ * completed steps.  A harness uses it to start the step-by-step comparison from a state that was
+ * reached elsewhere (a long warm-up that the oracle is too slow to follow).
+ */
+int mko_load_decode_state(mko_state *s, int g, int n, const double *K, const double *V,
+                          const double *I, const int64_t *pos, int64_t steps_done) {
+    if (g < 0 || g >= s->Hkv || n < 0 || s->pending) return -1;
+    mko_head *hd = &s->h[g];
+    head_reserve(hd, s->d, n + 1);
+    memcpy(hd->K, K, sizeof(double) * (size_t)n * s->d);
+    memcpy(hd->V, V, sizeof(double) * (size_t)n * s->d);
+    for (int i = 0; i < n; ++i) { hd->I[i] = I[i]; hd->pos[i] = pos[i]; hd->abar[i] = 0.0; }
+    hd->n = n;
+    hd->ev_n = 0;
+    s->t = steps_done;
+    return 0;
+}
+
+/*
  * Algorithm 1, from the append up to and including the importance update.
  * q [Hq][d], k_new, v_new [Hkv][d], out [Hq][d].
  */

@@ -46,6 +46,7 @@ def lib():
         L.mko_destroy.argtypes = [C.c_void_p]
         L.mko_prefill.argtypes = [C.c_void_p, dp, dp]
         L.mko_set_budget.argtypes = [C.c_void_p, C.c_int]
+        L.mko_load_decode_state.argtypes = [C.c_void_p, C.c_int, C.c_int, dp, dp, dp, lp, C.c_int64]
         L.mko_attend_update.argtypes = [C.c_void_p, dp, dp, dp, dp]
         L.mko_evict.argtypes = [C.c_void_p, lp, ip, C.c_int]
         L.mko_step.argtypes = [C.c_void_p, dp, dp, dp, dp]
@@ -112,6 +113,17 @@ class OracleSequence:
 
     def set_budget(self, budget):
         lib().mko_set_budget(self._h, int(budget))
+
+    def load_decode_state(self, g, K, V, score, pos, steps_done):
+        """Puts KV head g's decode pool into the given state (a loader: no arithmetic)."""
+        K, V, score = _f64(K), _f64(V), _f64(score)
+        pos = np.ascontiguousarray(pos, dtype=np.int64)
+        n = score.shape[0]
+        assert K.shape == (n, self.d) and V.shape == (n, self.d) and pos.shape == (n,)
+        rc = lib().mko_load_decode_state(self._h, g, n, _d(K), _d(V), _d(score),
+                                         pos.ctypes.data_as(C.POINTER(C.c_int64)), int(steps_done))
+        if rc:
+            raise RuntimeError(f"mko_load_decode_state rc={rc}")
 
     def attend_update(self, q, k_new, v_new):
         q, k_new, v_new = _f64(q), _f64(k_new), _f64(v_new)

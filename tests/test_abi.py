@@ -110,6 +110,10 @@ def test_start_table_invariants(lib):
             t0 = tiles.sum() * c // len(u0)
             assert begin[u0[c]] <= t0 < begin[u0[c] + 1]
         assert set(hn.tolist()) <= {0, 4}
+        # another reservation size: same spread, reserved ranges of that size
+        u0b, h0b, hnb, nxb, _ = mkv.plan_starts(B, hkv, budget, lens, nmax, head_tiles=7)
+        assert (u0b == u0).all() and set(hnb.tolist()) <= {0, 7} and (nxb % 7 == 0).all()
+        assert (mkv.plan_starts(B, hkv, budget, lens, nmax, head_tiles=0)[2] == 0).all()
         for u in range(U):
             mine = np.where(u0 == u)[0]
             got = sorted((int(h0[c]), int(hn[c])) for c in mine if hn[c] > 0)
@@ -118,3 +122,45 @@ def test_start_table_invariants(lib):
             assert nx[u] == 4 * len(got) <= -(-int(lens[u // hkv]) // 64)
             assert len(mine) <= 32 and ch[u] >= 2
             assert len(mine) + -(-int(tiles[u] - nx[u]) // int(ch[u])) <= 64 - 8
+
+
+def test_reproducible_mode_ranges_cover_every_tile_once(lib):
+    """mkv_plan_ranges: the CTAs' ranges tile the global tile sequence without gap or overlap,
+    a unit's partial slots (CTA index minus the unit's first CTA) are 0..visits-1 with at most 64
+    visits, and every CTA has work."""
+    import numpy as np
+    from workloads.synthetic import CONFIGS
+    cases = [(CONFIGS["llama_b16"].prefill_lens(), 8, 1024, 296), (np.array([64], dtype=np.int32), 1, 64, 296),
+             (np.array([0, 5, 4096], dtype=np.int32), 4, 128, 148), (np.full(64, 512, dtype=np.int32), 4, 2048, 296),
+             (np.array([100000], dtype=np.int32), 2, 16, 296), (np.array([0], dtype=np.int32), 1, 1, 296)]
+    for lens, hkv, budget, nmax in cases:
+        B, U = len(lens), len(lens) * hkv
+        t0, tb, uc = mkv.plan_ranges(B, hkv, budget, lens, nmax)
+        n = len(t0) - 1
+        tiles = np.array([-(-int(lens[u // hkv]) // 64) + -(-budget // 64) for u in range(U)])
+        assert (np.diff(tb) == tiles).all() and tb[0] == 0
+        assert 1 <= n <= nmax and t0[0] == 0 and t0[-1] == tiles.sum() and (np.diff(t0) >= 1).all()
+        for u in range(U):
+            touching = [c for c in range(n) if t0[c] < tb[u + 1] and t0[c + 1] > tb[u]]
+            assert touching == list(range(uc[u], uc[u] + len(touching))) and 1 <= len(touching) <= 64
+
+
+def test_grid_limit_clamps_to_what_is_resident(lib):
+    """The grid never exceeds SM count x resident CTAs per SM (the kernels' CTAs wait on one
+    another), never the design point, never 2048; a kernel that does not fit gives 0."""
+    assert mkv.grid_limit(148, 2, 2) == 296
+    assert mkv.grid_limit(148, 1, 2) == 148          # a deeper ring: one CTA per SM fits
+    assert mkv.grid_limit(148, 5, 2) == 296          # more would fit, the design point stands
+    assert mkv.grid_limit(148, 16, 8) == 1184
+    assert mkv.grid_limit(1000, 8, 8) == 2048
+    assert mkv.grid_limit(148, 0, 2) == 0 and mkv.grid_limit(0, 2, 2) == 0
+
+
+def test_new_calls_check_their_arguments(lib):
+    one = C.c_void_p(256)
+    assert lib.mkv_set_option(None, 1, 3) == 1
+    assert lib.mkv_decode_step_layers(None, 0, 1, one, one, one, one, None) == 1
+    assert lib.mkv_attend_only_layers(None, 0, 1, one, one, None) == 1
+    assert lib.mkv_debug_withhold_tile(None, 0, 0, 0) == 1
+    n, m = C.c_int32(0), C.c_int32(0)
+    assert lib.mkv_get_grid(None, 0, C.byref(n), C.byref(m)) == 1

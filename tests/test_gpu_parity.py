@@ -167,115 +167,6 @@ def test_two_layers_keep_independent_state():
         assert rep.steps == 120 and rep.evictions > 0
 
 
-def attention_f64(q, K, V, G):
-    """softmax(q K^T / sqrt(d)) V written out in numpy fp64; q [Hq,d], K/V [Hkv,N,d]."""
-    d = q.shape[-1]
-    out = np.zeros_like(q)
-    probs = []
-    for h in range(q.shape[0]):
-        s = K[h // G] @ q[h] / np.sqrt(d)
-        e = np.exp(s - s.max())
-        pr = e / e.sum()
-        probs.append(pr)
-        out[h] = pr @ V[h // G]
-    return out, probs
-
-
-FULL_SIZE_CASES = {
-    # name: (workload, layers, layer-wide score mode, sampled sequences)
-    "llama_b16": (lambda: CONFIGS["llama_b16"], 1, False, None),
-    "llama_b16_layer_mean": (lambda: CONFIGS["llama_b16"], 1, True, None),
-    "llama_stack_two_layers": (lambda: CONFIGS["llama_stack"], 2, False, None),
-    "qwen_b64_budget128_beta0.8": (lambda: CONFIGS["qwen_b64"].with_(budget=128, beta=0.8), 1, False, None),
-    "qwen_b64_budget1024_beta0.99": (lambda: CONFIGS["qwen_b64"].with_(budget=1024, beta=0.99), 1, False, None),
-}
-
-
-@pytest.mark.parametrize("case", sorted(FULL_SIZE_CASES))
-def test_full_size_sampled_units_at_steady_state(case):
-    """The benchmark configurations at their full sizes (batch, prefill lengths, budget, the grid
-    and chunking the bench times), run to steady state with device-generated inputs.  One further
-    step is then checked on sampled sequences against the definitions computed from the GPU's
-    own pre-step state: attention over prefill + pool + fresh token (Eq. 2), Eq. 4-5 scores in the
-    context's score mode, and the oracle's select() for the evicted token (Eq. 8)."""
-    import torch
-    from oracle import mkv_oracle as O
-    make_w, layers, layer_mean, _ = FULL_SIZE_CASES[case]
-    w = make_w()
-    lens = w.prefill_lens()
-    B, Hq, Hkv, d, G = w.batch, w.q_heads, w.kv_heads, w.head_dim, w.group
-    dev = torch.device("cuda", 0)
-    ctx = mkv.MomentKV(layers, Hq, Hkv, d, w.budget, w.beta, B, int(lens.max()), out_dtype=mkv.MKV_F32,
-                       score_mode=mkv.MKV_SCORE_LAYER_MEAN if layer_mean else mkv.MKV_SCORE_GROUP_MEAN)
-    gen = torch.Generator(device=dev)
-    gen.manual_seed(11)
-    for layer in range(layers):
-        K = (torch.randn((B, Hkv, int(lens.max()), d), generator=gen, device=dev) / d ** 0.5).bfloat16()
-        V = (torch.randn((B, Hkv, int(lens.max()), d), generator=gen, device=dev) / d ** 0.5).bfloat16()
-        ctx.prefill(layer, K, V, lens)
-        torch.cuda.synchronize()
-        del K, V
-    out = torch.zeros((B, Hq, d), dtype=torch.float32, device=dev)
-    ring = 32
-    qs = (2.0 * torch.randn((ring, B, Hq, d), generator=gen, device=dev)).bfloat16()
-    ks = (torch.randn((ring, B, Hkv, d), generator=gen, device=dev) / d ** 0.5).bfloat16()
-    vs = (torch.randn((ring, B, Hkv, d), generator=gen, device=dev) / d ** 0.5).bfloat16()
-    steps = w.budget + 40
-    for i in range(steps):
-        for layer in range(layers):
-            ctx.decode_step(layer, qs[(i + layer) % ring], ks[(i + layer) % ring], vs[(i + layer) % ring], out)
-    ctx.status_sync()
-    layer = layers - 1
-    seqs = sorted({0, B // 2, B - 1, int(np.argmax(lens)), int(np.argmin(lens))})
-    before = {}
-    for b in seqs:
-        for g in range(Hkv):
-            Kp, Vp = ctx.read_kv(layer, b, g, 0)
-            Kd, Vd = ctx.read_kv(layer, b, g, 1)
-            pos, sc = ctx.decode_state(layer, b, g)
-            assert len(pos) == w.budget
-            before[(b, g)] = (Kp, Vp, Kd, Vd, pos, sc)
-    i = steps + layer
-    ctx.decode_step(layer, qs[i % ring], ks[i % ring], vs[i % ring], out)
-    ctx.status_sync()
-    got = out.double().cpu().numpy()
-    qh = qs[i % ring].double().cpu().numpy()
-    kh = ks[i % ring].double().cpu().numpy()
-    vh = vs[i % ring].double().cpu().numpy()
-    for b in seqs:
-        head_probs = {}
-        for g in range(Hkv):
-            Kp, Vp, Kd, Vd, pos, sc = before[(b, g)]
-            Kall = np.concatenate([Kp, Kd, kh[b, g][None]])[None]
-            Vall = np.concatenate([Vp, Vd, vh[b, g][None]])[None]
-            ref, probs = attention_f64(qh[b, g * G:(g + 1) * G], Kall, Vall, G)
-            o = got[b, g * G:(g + 1) * G]
-            rowmax = np.abs(ref).max(axis=1, keepdims=True)
-            assert (np.abs(o - ref) <= 2e-3 * rowmax).all(), (b, g, np.abs(o - ref).max())
-            head_probs[g] = [pr[len(Kp):] for pr in probs]                     # decode slice, slot order
-        if layer_mean:   # every KV head's pool holds the same tokens in the same slots
-            for g in range(1, Hkv):
-                np.testing.assert_array_equal(before[(b, g)][4], before[(b, 0)][4])
-            abar_all = np.mean([pr for g in range(Hkv) for pr in head_probs[g]], axis=0)   # Eq. 4 over all H heads
-        for g in range(Hkv):
-            pos, sc = before[(b, g)][4], before[(b, g)][5]
-            abar = abar_all if layer_mean else np.mean(head_probs[g], axis=0)  # Eq. 4 over the KV group
-            new_sc = O.update(np.concatenate([sc.astype(np.float64), [0.0]]), abar, w.beta)   # Eq. 5, fresh token from 0
-            all_pos = np.concatenate([pos.astype(np.int64), [steps]])
-            pos2, sc2 = ctx.decode_state(layer, b, g)
-            ev_pos, ev_sc = ctx.last_evicted(layer, b, g)
-            assert len(pos2) == w.budget and len(ev_pos) == 1
-            g_pos = np.concatenate([pos2, ev_pos]).astype(np.int64)
-            g_sc = np.concatenate([sc2, ev_sc]).astype(np.float64)
-            assert sorted(g_pos.tolist()) == sorted(all_pos.tolist())
-            order, rorder = np.argsort(g_pos), np.argsort(all_pos)
-            rel = np.abs(g_sc[order] - new_sc[rorder]) / np.maximum(new_sc[rorder], 1e-300)
-            assert rel.max() <= 1e-4, (b, g, rel.max())
-            want = g_pos[O.select(g_sc, g_pos, 1)]        # integer selection on the GPU's own scores
-            assert want.tolist() == ev_pos.tolist()
-    ctx.close()
-
-
 @pytest.mark.parametrize("shape", ["llama_bf16", "small_f32"])
 def test_layer_mean_mode_scores_over_all_heads(shape):
     """MKV_SCORE_LAYER_MEAN with several KV heads (Eq. 4 as printed: the mean runs over all H

@@ -340,3 +340,37 @@ def test_forced_eviction_and_budget_shrink():
     pos, _, _ = o.decode_state(0)
     o.evict(force=[[int(pos[0])]])
     assert int(pos[0]) not in o.decode_state(0)[0] and o.count(0) == 4
+
+
+@pytest.mark.parametrize("mode", [O.GROUP_MEAN, O.LAYER_MEAN])
+def test_loaded_state_continues_like_the_uninterrupted_run(mode):
+    """The state loader holds no arithmetic: an oracle whose decode pools are loaded from
+    another oracle's state (in a different slot order: Algorithm 1 does not depend on the order
+    of the pool, and ties go by position id) continues with exactly the same evictions and, up
+    to summation order, the same outputs and scores."""
+    rng = np.random.default_rng(21)
+    Hq, Hkv, d, Lp, T0, T1, budget = 6, 2, 16, 9, 20, 12, 7
+    Kp, Vp, q, k, v = rand_problem(rng, Hq, Hkv, d, Lp, T0 + T1, scale=1.5)
+    a = O.OracleSequence(Hq, Hkv, d, budget, 0.85, Lp, mode)
+    a.prefill(Kp, Vp)
+    for t in range(T0):
+        a.step(q[t], k[t], v[t])
+    b = O.OracleSequence(Hq, Hkv, d, budget, 0.85, Lp, mode)
+    b.prefill(Kp, Vp)
+    perm = rng.permutation(budget)                           # the same order in every KV head
+    for g in range(Hkv):
+        pos, sc, _ = a.decode_state(g)
+        Kd, Vd = a.decode_kv(g)
+        b.load_decode_state(g, Kd[perm], Vd[perm], sc[perm], pos[perm], T0)
+    assert b.steps_done() == T0
+    for t in range(T0, T0 + T1):
+        oa, ob = a.attend_update(q[t], k[t], v[t]), b.attend_update(q[t], k[t], v[t])
+        np.testing.assert_allclose(ob, oa, rtol=1e-12, atol=1e-14)
+        for g in range(Hkv):
+            assert sorted(a.choose(g).tolist()) == sorted(b.choose(g).tolist())
+        a.evict(); b.evict()
+        for g in range(Hkv):
+            pa, sa, _ = a.decode_state(g)
+            pb, sb, _ = b.decode_state(g)
+            np.testing.assert_array_equal(np.sort(pa), np.sort(pb))
+            np.testing.assert_allclose(sb[np.argsort(pb)], sa[np.argsort(pa)], rtol=1e-12)
