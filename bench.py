@@ -9,6 +9,14 @@ at steady state, i.e. with the decode pool full so that every step evicts.  `--l
 identical layers are cycled so that every layer-step streams a cache that is cold in L2
 (as in a real 32-layer model).
 
+Timing.  The steps of a decode loop overlap (a step starts while the previous one ends), so
+a timed region must begin with the pipeline full: after the barrier + synchronize, a lead-in
+of untimed steps is enqueued, the first event is recorded behind it without any
+synchronisation, exactly K steps follow, then the second event and a barrier + synchronize.
+Plain attention on the same state (mkv_attend_only: the reference the score/evict overhead is
+quoted against) is timed the same way over the same number of steps; the two arms alternate
+for a few rounds and the medians are reported.
+
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl mkv|reference]
 
 prints one JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle instead.
@@ -34,7 +42,7 @@ ROW_BYTES = 512  # K + V bytes of one cached token of one KV head (d=128 bf16)
 
 # DRAM traffic of the hot kernel from its ncu capture (profiles/), as a ratio to the
 # algorithmic bytes of the captured case; valid only for the kernel sources it was taken on.
-TRAFFIC_CAPTURE = {"sources_sha1": "88090bc204f461ad5174750b8db4473649be547f", "traffic_over_algorithmic": 1.0260}
+TRAFFIC_CAPTURE = {"sources_sha1": "", "traffic_over_algorithmic": None}
 KERNEL_SOURCES = ["mkv_mma.cu", "mkv_tail.cuh", "mkv_layer_tail.cuh", "mkv_common.cuh", "mkv_ptx.cuh", "mkv_api.cu"]
 
 
@@ -208,7 +216,7 @@ def run_reference(args, w):
         "impl": "reference", "metric": "decode tokens/sec per layer", "value": value, "unit": "tokens/s",
         "n_gpus": args.gpus, "steps": done["timed"], "warmup": done["warm"], "ms_per_step": 1e3 * w.batch / value,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(w, lens, args),
+        "config": workload_config(w, lens, args, args.inputs),
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -216,7 +224,7 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
-def workload_config(w, lens, args):
+def workload_config(w, lens, args, inputs="plain", older=None):
     shape = {"llama_b16": "Llama-3.1-8B attention layer shape", "llama_b1": "Llama-3.1-8B attention layer shape",
              "llama_stack": "Llama-3.1-8B attention layer shape", "qwen_b64": "Qwen2.5-7B-like attention layer shape",
              "tiny": "tiny single-layer shape"}.get(w.name, w.name)
@@ -224,10 +232,23 @@ def workload_config(w, lens, args):
     return {"workload": f"{w.name}: {shape}, {w.q_heads}/{w.kv_heads} heads, "
                         f"head_dim {w.head_dim}, {w.dtype}, batch {w.batch}, {pre} "
                         f"(sum {int(np.sum(lens))}), decode budget {w.budget}, beta {w.beta}, steady state "
-                        f"(decode pool full, one eviction per unit per step)",
+                        f"(decode pool full, one eviction per unit per step); " + input_note(inputs, older),
             "layers_cycled": args.layers,
             "l2": "inputs larger than L2: each layer-step streams its own ~%d MB cache, %d layers cycled"
                   % (int(sum(w.kv_heads * (int(lp) + w.budget + 1) * 2 * w.head_dim * (2 if w.dtype == "bf16" else 4) for lp in lens) / 1e6), args.layers)}
+
+
+def input_note(inputs, older):
+    if inputs == "hot":
+        note = ("device-generated inputs of the 'hot' kind: queries 2*sqrt(d)*N(0,1), keys N(0,1)/sqrt(d) plus half a "
+                "unit vector along the group's mean query, values N(0,1)/sqrt(d), so that evictions hit tokens of all "
+                "ages and the fresh row is stored into the evicted slot")
+    else:
+        note = ("device-generated N(0,1) queries and N(0,1)/sqrt(d) keys and values: attention is near uniform and the "
+                "token evicted is almost always the fresh one, whose row is then not stored")
+    if older is not None:
+        note += f" (in the last timed step {older[0]} of {older[1]} units evicted an older token)"
+    return note
 
 
 def rank_workload(w, rank):
@@ -251,27 +272,180 @@ def job_tokens_per_s(batch, steps, world, ms_max):
     return world * batch * steps / (ms_max * 1e-3)
 
 
+
+def make_ring(torch, gen, ring, lead, Hq, Hkv, d, tdt, dev, inputs):
+    """A ring of pre-generated step inputs on the device: q [ring, *lead, Hq, d], k_new / v_new
+    [ring, *lead, Hkv, d].  They are final before any step is enqueued."""
+    G = Hq // Hkv
+    z = torch.randn((ring, *lead, Hq, d), generator=gen, device=dev)
+    k = torch.randn((ring, *lead, Hkv, d), generator=gen, device=dev) / d ** 0.5
+    v = torch.randn((ring, *lead, Hkv, d), generator=gen, device=dev) / d ** 0.5
+    if inputs == "hot":
+        q = 2.0 * d ** 0.5 * z
+        qbar = q.reshape(ring, *lead, Hkv, G, d).mean(dim=-2)
+        k = k + 0.5 * qbar / qbar.norm(dim=-1, keepdim=True)
+    else:
+        q = z
+    return q.to(tdt).contiguous(), k.to(tdt).contiguous(), v.to(tdt).contiguous()
+
+
+class Arm:
+    """One configuration set up on the device at steady state: context, input ring, step functions."""
+
+    def __init__(self, torch, mkv, w, lens, layers, dev, seed, inputs, score_mode="group", kernel="auto", stacked=False,
+                 out_dtype=None, head_tiles=None, fill=None, early=True):
+        self.torch, self.w, self.layers, self.stacked = torch, w, layers, stacked
+        B, Hq, Hkv, d = w.batch, w.q_heads, w.kv_heads, w.head_dim
+        kv_dtype = mkv.MKV_BF16 if w.dtype == "bf16" else mkv.MKV_F32
+        tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+        Lmax = int(lens.max())
+        self.ctx = mkv.MomentKV(layers, Hq, Hkv, d, w.budget, w.beta, B, Lmax, kv_dtype=kv_dtype,
+                                out_dtype=kv_dtype if out_dtype is None else out_dtype,
+                                kernel={"auto": mkv.MKV_KERNEL_AUTO, "simt": mkv.MKV_KERNEL_SIMT, "mma": mkv.MKV_KERNEL_MMA}[kernel],
+                                device=dev.index,
+                                score_mode=mkv.MKV_SCORE_LAYER_MEAN if score_mode == "layer" else mkv.MKV_SCORE_GROUP_MEAN,
+                                flags=mkv.MKV_FLAG_INPUTS_READY if early else 0)
+        if head_tiles is not None:
+            self.ctx.set_option(mkv.MKV_OPT_HEAD_TILES, head_tiles)
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(seed)
+        for layer in range(layers):
+            K = (torch.randn((B, Hkv, Lmax, d), generator=gen, device=dev) / d ** 0.5).to(tdt)
+            V = (torch.randn((B, Hkv, Lmax, d), generator=gen, device=dev) / d ** 0.5).to(tdt)
+            self.ctx.prefill(layer, K, V, lens)
+            torch.cuda.synchronize()
+            del K, V
+        self.ring = 8 if stacked else 64
+        lead = (layers, B) if stacked else (B,)
+        self.qs, self.ks, self.vs = make_ring(torch, gen, self.ring, lead, Hq, Hkv, d, tdt, dev, inputs)
+        odt = torch.float32 if (out_dtype is not None and out_dtype == mkv.MKV_F32) else tdt
+        self.out = torch.empty((*lead, Hq, d), dtype=odt, device=dev)
+        torch.cuda.synchronize()
+        self.per_call = layers if stacked else 1        # layer-steps one call performs
+        self.fill_steps = w.budget if fill is None else fill
+
+    def step(self, i):
+        r = i % self.ring
+        if self.stacked:
+            self.ctx.decode_step_layers(0, self.layers, self.qs[r], self.ks[r], self.vs[r], self.out)
+        else:
+            self.ctx.decode_step(i % self.layers, self.qs[r], self.ks[r], self.vs[r], self.out)
+
+    def attend(self, i):
+        r = i % self.ring
+        if self.stacked:
+            self.ctx.attend_only_layers(0, self.layers, self.qs[r], self.out)
+        else:
+            self.ctx.attend_only(i % self.layers, self.qs[r], self.out)
+
+    def fill(self, stream, timed=False):
+        """Every layer's decode pool from empty to `fill_steps` tokens; returns ms per layer-step."""
+        torch = self.torch
+        n = self.fill_steps * (1 if self.stacked else self.layers)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for i in range(10):
+            self.attend(i)                               # warms the kernel up; leaves the state alone
+        torch.cuda.synchronize()
+        ev0.record(stream)
+        for i in range(n):
+            self.step(i)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        self.ctx.status_sync()
+        return ev0.elapsed_time(ev1) / (n * self.per_call)
+
+    def close(self):
+        self.ctx.close()
+
+
+def timed_rounds(torch, stream, barrier, arm, calls, lead_in, rounds, with_attend=True):
+    """`rounds` times: [lead-in, event, `calls` decode calls, event] then the same with plain
+    attention.  Returns per-round ms per call for both arms and the launches of one timed part."""
+    dec, att = [], []
+    launches = 0
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    i = 0
+    for _ in range(rounds):
+        barrier()
+        for _ in range(lead_in):
+            arm.step(i); i += 1
+        l0 = arm.ctx.launch_count()
+        ev[0].record(stream)
+        for _ in range(calls):
+            arm.step(i); i += 1
+        ev[1].record(stream)
+        launches = arm.ctx.launch_count() - l0
+        if with_attend:
+            for j in range(lead_in):
+                arm.attend(j)
+            ev[2].record(stream)
+            for j in range(calls):
+                arm.attend(j)
+            ev[3].record(stream)
+        barrier()
+        dec.append(ev[0].elapsed_time(ev[1]) / calls)
+        if with_attend:
+            att.append(ev[2].elapsed_time(ev[3]) / calls)
+    return dec, att, launches
+
+
+def median(xs):
+    s = sorted(xs)
+    return s[len(s) // 2]
+
+
+def side_run(torch, mkv, stream, barrier, peak, w, lens, layers, dev, seed, inputs, name, calls=200, rounds=3, **kw):
+    """A short steady-state run of another configuration: one entry of `other_configs` / `comparison`."""
+    arm = Arm(torch, mkv, w, lens, layers, dev, seed, inputs, **kw)
+    ms_fill = arm.fill(stream)
+    for i in range(20):
+        arm.step(i)
+    dec, att, _ = timed_rounds(torch, stream, barrier, arm, calls, 50, rounds)
+    arm.ctx.status_sync()
+    n_dec = int(arm.ctx.decode_state(0, 0, 0)[0].shape[0])
+    arm.close()
+    ms = median(dec) / arm.per_call
+    ms_att = median(att) / arm.per_call
+    alg = algorithmic_bytes_per_step(w, lens, min(n_dec + 1, w.budget + 1), 1 if n_dec >= w.budget else 0)
+    gbs = alg / (ms * 1e-3) / 1e9
+    return {"name": name, "layers_per_launch": arm.per_call, "decode_pool_tokens": n_dec, "ms_per_layer_step": ms,
+            "tokens_per_s": w.batch / (ms * 1e-3), "algorithmic_bytes_per_step": alg, "achieved_gbs": gbs,
+            "frac": gbs / peak, "frac_of_nominal_8TBs": gbs / 8000.0, "attend_only_ms": ms_att,
+            "overhead_ratio": median([d / a for d, a in zip(dec, att)]), "ramp_ms_per_layer_step": ms_fill,
+            "steps_timed": calls, "rounds": rounds}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10000)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="mkv", choices=["mkv", "reference"])
     ap.add_argument("--config", default="llama_b16", choices=sorted(CONFIGS))
-    ap.add_argument("--layers", type=int, default=4)
+    ap.add_argument("--layers", type=int, default=0, help="layers cycled (0: 4, or the whole stack for llama_stack)")
     ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "mma"])
     ap.add_argument("--score-mode", default="group", choices=["group", "layer"],
                     help="group: mean over the query heads of a KV head (headline); layer: Eq. 4 over all heads")
     ap.add_argument("--budget", type=int, default=0, help="override the workload's decode budget (profiling small cases)")
+    ap.add_argument("--inputs", default="hot", choices=["hot", "plain"], help="kind of device-generated step inputs")
+    ap.add_argument("--head-tiles", type=int, default=-1, help="reserved prompt tiles per CTA (default: the library's)")
+    ap.add_argument("--no-early", action="store_true", help="do not promise that the inputs are final at enqueue time")
+    ap.add_argument("--per-layer", action="store_true", help="llama_stack: one launch per layer instead of one per stack")
+    ap.add_argument("--rounds", type=int, default=5)
+    ap.add_argument("--lead-in", type=int, default=200)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay timing")
+    ap.add_argument("--no-others", action="store_true", help="skip the other configurations and the comparison runs")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     w = CONFIGS[args.config]
     if args.budget > 0:
         w = w.with_(budget=args.budget)
+    stacked = args.config == "llama_stack" and not args.per_layer
+    if args.layers <= 0:
+        args.layers = w.layers if args.config == "llama_stack" else 4
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -290,118 +464,69 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    # every rank holds its own batch (weak scaling; units are independent, no collective)
-    wr = rank_workload(w, rank)
-    lens = wr.prefill_lens()
-    Lmax = int(lens.max())
-    B, Hq, Hkv, d = w.batch, w.q_heads, w.kv_heads, w.head_dim
-    kernel = {"auto": mkv.MKV_KERNEL_AUTO, "simt": mkv.MKV_KERNEL_SIMT, "mma": mkv.MKV_KERNEL_MMA}[args.kernel]
-    kv_dtype = mkv.MKV_BF16 if w.dtype == "bf16" else mkv.MKV_F32
-    tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
-    ctx = mkv.MomentKV(args.layers, Hq, Hkv, d, w.budget, w.beta, B, Lmax, kv_dtype=kv_dtype, out_dtype=kv_dtype,
-                       kernel=kernel, device=local,
-                       score_mode=mkv.MKV_SCORE_LAYER_MEAN if args.score_mode == "layer" else mkv.MKV_SCORE_GROUP_MEAN)
-    gen = torch.Generator(device=dev)
-    gen.manual_seed(1234 + rank)
-    for layer in range(args.layers):
-        K = (torch.randn((B, Hkv, Lmax, d), generator=gen, device=dev) / d ** 0.5).to(tdt)
-        V = (torch.randn((B, Hkv, Lmax, d), generator=gen, device=dev) / d ** 0.5).to(tdt)
-        ctx.prefill(layer, K, V, lens)
-        torch.cuda.synchronize()
-        del K, V
-    ring = 64
-    qs = torch.randn((ring, B, Hq, d), generator=gen, device=dev).to(tdt)
-    ks = (torch.randn((ring, B, Hkv, d), generator=gen, device=dev) / d ** 0.5).to(tdt)
-    vs = (torch.randn((ring, B, Hkv, d), generator=gen, device=dev) / d ** 0.5).to(tdt)
-    out = torch.empty((B, Hq, d), dtype=tdt, device=dev)
-
-    def step(i):
-        ctx.decode_step(i % args.layers, qs[i % ring], ks[i % ring], vs[i % ring], out)
-
-    stream = torch.cuda.current_stream(dev)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    # The ramp: every layer's decode pool from empty to the budget, timed on its own (steps get
-    # longer as the pool grows); it also is the set-up of the steady state measured below.
-    # Plain attention launches warm the kernel up first: they leave the state alone.
-    for i in range(10):
-        ctx.attend_only(i % args.layers, qs[i % ring], out)
-    torch.cuda.synchronize()
-    n_ramp = w.budget * args.layers
-    ev0.record(stream)
-    for i in range(n_ramp):
-        step(i)
-    ev1.record(stream)
-    torch.cuda.synchronize()
-    ms_ramp = ev0.elapsed_time(ev1) / n_ramp
-    ctx.status_sync()
-    for i in range(args.warmup):
-        step(i)
-    sampler = ClockSampler(local)
-
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    barrier()
-    launches0 = ctx.launch_count()
+    # every rank holds its own batch (weak scaling; units are independent, no collective)
+    wr = rank_workload(w, rank)
+    lens = wr.prefill_lens()
+    B, Hq, Hkv, d = w.batch, w.q_heads, w.kv_heads, w.head_dim
+    tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    head_tiles = args.head_tiles if args.head_tiles >= 0 else None
+    arm = Arm(torch, mkv, w, lens, args.layers, dev, 1234 + rank, args.inputs, score_mode=args.score_mode,
+              kernel=args.kernel, stacked=stacked, head_tiles=head_tiles, early=not args.no_early)
+    ctx = arm.ctx
+    stream = torch.cuda.current_stream(dev)
+    # The ramp: every layer's decode pool from empty to the budget, timed on its own (steps get
+    # longer as the pool grows); it also is the set-up of the steady state measured below.
+    ms_ramp = arm.fill(stream)
+    for i in range(args.warmup):
+        arm.step(i)
+    sampler = ClockSampler(local)
+    calls = max(1, args.steps // arm.per_call) if stacked else args.steps
     sampler.start()
-    # five equal segments of the timed region get events of their own (spread of the step time)
-    n_seg = 5 if args.steps >= 50 else 1
-    seg_ev = [torch.cuda.Event(enable_timing=True) for _ in range(n_seg - 1)]
-    seg_at = {args.steps * (j + 1) // n_seg: seg_ev[j] for j in range(n_seg - 1)}
-    ev0.record(stream)
-    for i in range(args.steps):
-        step(i)
-        if i + 1 in seg_at:
-            seg_at[i + 1].record(stream)
-    ev1.record(stream)
-    barrier()
+    dec, att, launches = timed_rounds(torch, stream, barrier, arm, calls, args.lead_in, max(1, args.rounds))
     clocks = sampler.stop()
-    launches = ctx.launch_count() - launches0
-    ms = ev0.elapsed_time(ev1)
-    marks = [ev0] + seg_ev + [ev1]
-    bounds = [0] + sorted(seg_at) + [args.steps]
-    seg_ms = [marks[j].elapsed_time(marks[j + 1]) / max(bounds[j + 1] - bounds[j], 1) for j in range(n_seg)]
     ctx.status_sync()
-
-    # plain decode attention on the same state (no append/score/evict): overhead reference
-    for i in range(10):
-        ctx.attend_only(i % args.layers, qs[i % ring], out)
-    barrier()
-    n_att = max(100, args.steps // 4)
-    ev0.record(stream)
-    for i in range(n_att):
-        ctx.attend_only(i % args.layers, qs[i % ring], out)
-    ev1.record(stream)
-    barrier()
-    ms_att = ev0.elapsed_time(ev1) / n_att
+    # which tokens the last timed step evicted (the fresh one, or an older one whose slot took the fresh row)
+    older = [0, 0]
+    for b in range(B):
+        for g in range(Hkv):
+            ev_pos, _ = ctx.last_evicted(0, b, g)
+            if len(ev_pos):
+                older[1] += 1
+                older[0] += int(int(ev_pos[0]) != ctx.step_count(0) - 1)
 
     # the same steps recorded once and replayed as a CUDA graph (what a serving loop would do):
     # launch cost leaves the host, which shows on the small, launch-bound workloads
-    ms_graph, n_rec = 0.0, 16 * args.layers
+    ms_graph, n_rec = 0.0, (4 if stacked else 16 * args.layers)
     if not args.no_graph:
         side = torch.cuda.Stream(dev)
         side.wait_stream(stream)
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=side):
             for i in range(n_rec):
-                step(i)
-        reps = max(3, args.steps // n_rec)
+                arm.step(i)
+        reps = max(3, calls // n_rec)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
         for _ in range(3):
             graph.replay()
-        barrier()
         ev0.record(stream)
         for _ in range(reps):
             graph.replay()
         ev1.record(stream)
         barrier()
-        ms_graph = ev0.elapsed_time(ev1) / (reps * n_rec)
+        ms_graph = ev0.elapsed_time(ev1) / (reps * n_rec * arm.per_call)
         ctx.status_sync()
 
     # end to end through the host-buffer entry point: H2D of q,k,v and D2H of out every step
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not stacked:
+        qs, ks, vs = arm.qs, arm.ks, arm.vs
+        ring = arm.ring
         # one pinned buffer per step holding q | k_new | v_new back to back (a single H2D copy)
         nq, nk = qs[0].numel(), ks[0].numel()
         packed = torch.empty((ring, nq + 2 * nk), dtype=tdt).pin_memory()
@@ -412,10 +537,11 @@ def main():
         hk = [packed[i, nq:nq + nk] for i in range(ring)]
         hv = [packed[i, nq + nk:] for i in range(ring)]
         hout = torch.empty((B, Hq, d), dtype=tdt).pin_memory()
-        n_e2e = max(100, args.steps // 4)
+        n_e2e = max(100, min(args.steps, 2000))
         for i in range(10):
             ctx.decode_step_host(i % args.layers, hq[i % ring], hk[i % ring], hv[i % ring], hout)
             stream.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         ev0.record(stream)
         for i in range(n_e2e):
@@ -423,35 +549,49 @@ def main():
             stream.synchronize()          # the host reads the step's result before the next step
         ev1.record(stream)
         barrier()
-        ms_e2e = ev0.elapsed_time(ev1)
         es = qs.element_size()
-        e2e = {"ms": ms_e2e, "steps": n_e2e, "h2d": (qs[0].numel() + ks[0].numel() + vs[0].numel()) * es,
+        e2e = {"ms": ev0.elapsed_time(ev1), "steps": n_e2e, "h2d": (qs[0].numel() + ks[0].numel() + vs[0].numel()) * es,
                "d2h": hout.numel() * hout.element_size()}
+    arm.close()
 
-    ms_max, ms_att_max, ms_e2e_max, ms_ramp_max, ms_graph_max = max_over_ranks(
-        [ms, ms_att, e2e["ms"] / e2e["steps"] if e2e else 0.0, ms_ramp, ms_graph], world, dev)
+    R = len(dec)
+    red = max_over_ranks(dec + att + [e2e["ms"] / e2e["steps"] if e2e else 0.0, ms_ramp, ms_graph], world, dev)
+    dec_max, att_max = red[:R], red[R:2 * R]
+    ms_e2e_max, ms_ramp_max, ms_graph_max = red[2 * R:]
 
     if rank == 0:
-        ms_per_step = ms_max / args.steps
-        tokens_per_s = job_tokens_per_s(B, args.steps, world, ms_max)
+        ms_call = median(dec_max)
+        ms_per_step = ms_call / arm.per_call                      # per layer-step
+        ms_att = median(att_max) / arm.per_call
+        tokens_per_s = world * B / (ms_per_step * 1e-3)
         peak, peak_kind = load_peaks()
         alg = algorithmic_bytes_per_step(w, lens, w.budget + 1, 1)
         achieved = alg / (ms_per_step * 1e-3) / 1e9
+        cfg = workload_config(w, lens, args, args.inputs, older)
+        cfg["launch"] = (f"one launch per {arm.per_call}-layer stack" if stacked else "one launch per layer-step")
+        cfg["early_inputs"] = not args.no_early
         line = {
             "metric": "decode tokens/sec per layer", "value": tokens_per_s, "unit": "tokens/s",
-            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "n_gpus": world, "steps": calls * arm.per_call, "warmup": args.warmup, "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w.dtype,
-            "data": "synthetic (device-generated N(0,1) queries, N(0,1)/sqrt(d) keys and values; shapes, "
-                    "lengths and budget of the named workload)",
-            "config": workload_config(w, lens, args),
-            "steps_per_s": world * args.steps / (ms_max * 1e-3),
+            "data": "synthetic (device-generated; shapes, lengths and budget of the named workload)",
+            "config": cfg,
+            "steps_per_s": world / (ms_per_step * 1e-3),
             "gpu_launches": int(launches),
             "clocks": clocks,
+            "timing": {"how": "barrier + synchronize, an untimed lead-in, event, the timed steps, event, barrier + "
+                              "synchronize; decode and plain attention alternate; medians over the rounds",
+                       "rounds": R, "lead_in_steps": args.lead_in, "timed_calls_per_round": calls,
+                       "layer_steps_per_call": arm.per_call,
+                       "ms_per_step_rounds": [x / arm.per_call for x in dec_max],
+                       "attend_only_ms_rounds": [x / arm.per_call for x in att_max]},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_kind": peak_kind, "frac_of_nominal_8TBs": achieved / 8000.0,
                          "algorithmic_bytes_per_step": alg, "traffic": captured_traffic(alg),
                          "kernel": "mma_kernel" if ctx_uses_mma(args, w) else "simt_kernel"},
-            "attend_only": {"ms_per_step": ms_att_max, "overhead_ratio": ms_per_step / ms_att_max},
+            "attend_only": {"ms_per_step": ms_att,
+                            "overhead_ratio": median([a / b for a, b in zip(dec_max, att_max)]),
+                            "how": "same state, same number of steps, same lead-in; median over the rounds of decode / plain"},
         }
         # whole run of the workload (its step count per layer): the measured ramp, then steady state
         T = max(int(w.steps), 1)
@@ -462,18 +602,16 @@ def main():
         line["whole_run"] = {"steps_per_layer": T, "ms_per_step": run_ms / T,
                              "tokens_per_s": world * B * T / (run_ms * 1e-3),
                              "how": "measured ramp mean x fill steps + measured steady state x the rest"}
-        if world == 1:
-            srt = sorted(seg_ms)
-            line["segments"] = {"n": n_seg, "median_ms_per_step": srt[len(srt) // 2], "min_ms_per_step": srt[0],
-                                "max_ms_per_step": srt[-1]}
         if ms_graph_max > 0.0:
-            line["graph_replay"] = {"ms_per_step": ms_graph_max, "steps_per_graph": n_rec,
+            line["graph_replay"] = {"ms_per_step": ms_graph_max, "steps_per_graph": n_rec * arm.per_call,
                                     "tokens_per_s": world * B / (ms_graph_max * 1e-3)}
         if e2e:
             line["e2e"] = {"value": world * B / (ms_e2e_max * 1e-3), "unit": "tokens/s",
                            "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                            "ms_per_step": ms_e2e_max, "sync": "stream synchronised after every step",
                            "how": "per step the GPU fetches q|k_new|v_new from the pinned host buffer (a small kernel ahead of the step) and the step's kernel writes out into the pinned host buffer"}
+        if world == 1 and not args.no_others and args.config == "llama_b16" and args.budget == 0:
+            line["other_configs"], line["comparison"] = other_runs(torch, mkv, stream, barrier, peak, dev, args)
         if not args.no_cpu_baseline and world == 1:
             n_units = min(len(os.sched_getaffinity(0)), B * Hkv)
             v, threads, sample, _ = time_oracle(w, lens, n_units, steps=48, warmup=2, time_cap_s=40.0, min_time_s=12.0)
@@ -481,6 +619,39 @@ def main():
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def other_runs(torch, mkv, stream, barrier, peak, dev, args):
+    """Short steady-state runs of the other configurations, and the comparison of the paper's
+    throughput figure (Sec. 7.4: full cache against score-tracking methods) inside the library:
+    the headline batch with a decode pool that is never evicted from, at the sizes a full cache
+    reaches after 4096 and 8192 generated tokens, against the budget of 1024; and the two limits
+    of the momentum factor (beta changes no byte that moves)."""
+    inputs = args.inputs
+    others = []
+    ws = CONFIGS["llama_stack"]
+    others.append(side_run(torch, mkv, stream, barrier, peak, ws, ws.prefill_lens(), ws.layers, dev, 21, inputs,
+                           "llama_stack: 32 layers, batch 4, prefill 2048, budget 2048; one launch per stack",
+                           calls=40, rounds=3, stacked=True))
+    for budget in (128, 1024):
+        wq = CONFIGS["qwen_b64"].with_(budget=budget)
+        others.append(side_run(torch, mkv, stream, barrier, peak, wq, wq.prefill_lens(), 4, dev, 22, inputs,
+                               f"qwen_b64: 28/4 heads (group 7), batch 64, prefill 512, budget {budget}", calls=400))
+    wl = CONFIGS["llama_b16"]
+    others.append(side_run(torch, mkv, stream, barrier, peak, wl, wl.prefill_lens(), 4, dev, 23, inputs,
+                           "llama_b16 in the score mode LAYER_MEAN (Eq. 4 over all heads of the layer)", calls=400,
+                           score_mode="layer"))
+    comparison = []
+    for pool in (4096, 8192):
+        wf = wl.with_(budget=pool + 2048)               # never reached: the pool only grows (full cache)
+        comparison.append(side_run(torch, mkv, stream, barrier, peak, wf, wf.prefill_lens(), 2, dev, 24, inputs,
+                                   f"full cache (no eviction), decode pool grown to about {pool} tokens", calls=100,
+                                   rounds=3, fill=pool - 300))
+    for beta in (0.0, 1.0):
+        wb = wl.with_(beta=beta)
+        comparison.append(side_run(torch, mkv, stream, barrier, peak, wb, wb.prefill_lens(), 2, dev, 25, inputs,
+                                   f"budget 1024, beta {beta}", calls=200, rounds=3))
+    return others, comparison
 
 
 def ctx_uses_mma(args, w):

@@ -80,13 +80,16 @@ def prefill_both(ctx, w: Workload, stream: BatchStream, layer=0, mode=O.GROUP_ME
 
 
 def lockstep(ctx, w: Workload, stream: BatchStream, oracles, steps, layer=0, report: ParityReport | None = None,
-             check_state_every=1, chunk=64, host_api=False, host_packed=False, host_pinned=True):
-    """Runs `steps` decode steps on both sides, comparing as described in the module doc."""
+             check_state_every=1, chunk=64, host_api=False, host_packed=False, host_pinned=True, tol_out=None,
+             tol_score=1e-4):
+    """Runs `steps` decode steps on both sides, comparing as described in the module doc.
+    tol_out / tol_score replace the standard tolerances (only the test of extreme logits does)."""
     torch = ctx.torch
     rep = report or ParityReport()
     B = len(oracles)
     dt, odt = ctx.torch_kv_dtype(), ctx.torch_out_dtype()
-    tol_out = 1e-5 if w.dtype == "f32" else 2e-3
+    if tol_out is None:
+        tol_out = 1e-5 if w.dtype == "f32" else 2e-3
     out = torch.zeros((B, w.q_heads, w.head_dim), dtype=odt, device=ctx.device)
     done = 0
     while done < steps:
@@ -147,7 +150,7 @@ def lockstep(ctx, w: Workload, stream: BatchStream, oracles, steps, layer=0, rep
                         sdiff = np.abs(all_sc[order] - o_sc[oorder])
                         serr = np.maximum(sdiff - FLUSH_ATOL, 0.0) / np.maximum(o_sc[oorder], 1e-300)
                         rep.max_score_err = max(rep.max_score_err, float(serr.max()))
-                        if serr.max() > 1e-4:
+                        if serr.max() > tol_score:
                             rep.failures.append(f"step {t} unit ({b},{g}): score error {serr.max():.3e}")
                         # teacher-forced: integer selection on the GPU's own scores
                         k = len(ev_pos)
