@@ -319,7 +319,9 @@ class Arm:
         lead = (layers, B) if stacked else (B,)
         self.qs, self.ks, self.vs = make_ring(torch, gen, self.ring, lead, Hq, Hkv, d, tdt, dev, inputs)
         odt = torch.float32 if (out_dtype is not None and out_dtype == mkv.MKV_F32) else tdt
-        self.out = torch.empty((*lead, Hq, d), dtype=odt, device=dev)
+        # neighbouring steps on different layers may run side by side: they get different outputs
+        self.outs = [torch.empty((*lead, Hq, d), dtype=odt, device=dev) for _ in range(2)]
+        self.out = self.outs[0]
         torch.cuda.synchronize()
         self.per_call = layers if stacked else 1        # layer-steps one call performs
         self.fill_steps = w.budget if fill is None else fill
@@ -327,16 +329,16 @@ class Arm:
     def step(self, i):
         r = i % self.ring
         if self.stacked:
-            self.ctx.decode_step_layers(0, self.layers, self.qs[r], self.ks[r], self.vs[r], self.out)
+            self.ctx.decode_step_layers(0, self.layers, self.qs[r], self.ks[r], self.vs[r], self.outs[i & 1])
         else:
-            self.ctx.decode_step(i % self.layers, self.qs[r], self.ks[r], self.vs[r], self.out)
+            self.ctx.decode_step(i % self.layers, self.qs[r], self.ks[r], self.vs[r], self.outs[i & 1])
 
     def attend(self, i):
         r = i % self.ring
         if self.stacked:
-            self.ctx.attend_only_layers(0, self.layers, self.qs[r], self.out)
+            self.ctx.attend_only_layers(0, self.layers, self.qs[r], self.outs[i & 1])
         else:
-            self.ctx.attend_only(i % self.layers, self.qs[r], self.out)
+            self.ctx.attend_only(i % self.layers, self.qs[r], self.outs[i & 1])
 
     def fill(self, stream, timed=False):
         """Every layer's decode pool from empty to `fill_steps` tokens; returns ms per layer-step."""

@@ -102,9 +102,15 @@ typedef enum {
                                     on any stream writes them.  A step may then begin its
                                     attention over the frozen prompt rows while the previous
                                     kernel of the stream (normally the previous step) is still
-                                    finishing.  Without the flag a step reads q only after every
-                                    earlier kernel of the stream has completed.  (The *_host
-                                    entry points ignore the flag.)                           */
+                                    finishing.  And a step whose layers are all different from
+                                    those of the context's previous step on the same stream
+                                    shares nothing with it (layers are independent instances of
+                                    Algorithm 1): it runs alongside that step from its start and
+                                    only its end is ordered behind it, so steps still complete
+                                    in stream order.  Such neighbours must therefore be given
+                                    different `out` buffers.  Without the flag a step reads q
+                                    only after every earlier kernel of the stream has completed.
+                                    (The *_host entry points ignore the flag.)               */
 #define MKV_FLAG_REPRODUCIBLE 4u /* same inputs, same bits: work is split among the CTAs by a
                                     fixed table instead of run-time counters and partial results
                                     are combined in a fixed order.  Costs some load balance;
@@ -348,14 +354,22 @@ int64_t mkv_launch_count(const mkv_ctx* ctx);
 mkv_status mkv_get_grid(const mkv_ctx* ctx, int layer, int32_t* n_ctas, int32_t* n_ctas_max);
 
 /*
- * Test hook for the error path of the bounded waits: one tile of unit (b, kv_head) of `layer`
- * counts as never delivered from now on, so the unit's finishing part, in the next step of that
- * layer, waits until the wait limit, gives up and sets MKV_ERR_TIMEOUT (nothing traps, nothing
- * spins without bound; the rest of the step completes).  The layer's results are undefined
- * afterwards: call mkv_reset() and prefill again.  Tensor-core kernel only (the scalar kernel
- * has no waits): otherwise MKV_ERR_UNSUPPORTED.  Synchronises the device.
+ * Test hooks for the kernels' error paths; nothing here traps, faults or spins without bound.
+ * Both act on the tensor-core kernel (otherwise MKV_ERR_UNSUPPORTED), synchronise the device, and
+ * leave the layer's results undefined: call mkv_reset() and prefill again afterwards.
+ *   MKV_INJECT_LOST_TILE          one tile of unit (b, kv_head) counts as never delivered: the
+ *                                 unit's finishing part never becomes due, which the last CTA of
+ *                                 the layer's next step notices on its way out
+ *                                 (MKV_ERR_DEVICE_CHECK; no waiting involved).
+ *   MKV_INJECT_EMPTY_QUEUE_ENTRY  the queue through which finished units reach idle CTAs claims
+ *                                 an entry that is never written: in the layer's next step a CTA
+ *                                 takes it, waits for its content up to the wait limit
+ *                                 (MKV_OPT_WAIT_LIMIT_US), gives up and sets MKV_ERR_TIMEOUT; the
+ *                                 rest of the step completes.  (b, kv_head are ignored.)
  */
-mkv_status mkv_debug_withhold_tile(mkv_ctx* ctx, int layer, int b, int kv_head);
+#define MKV_INJECT_LOST_TILE 0
+#define MKV_INJECT_EMPTY_QUEUE_ENTRY 1
+mkv_status mkv_debug_inject(mkv_ctx* ctx, int layer, int what, int b, int kv_head);
 
 /*
  * Recency-window attention diagnostics of the last decode step of `layer` (the analysis of

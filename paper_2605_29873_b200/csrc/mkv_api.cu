@@ -32,18 +32,20 @@ struct StateOff {
 };
 // Scratch that lives for one step only, shared by all launches of the context (calls on a
 // context are ordered on one stream, and a step touches it only after every earlier kernel
-// of the stream has completed).  Sized for a launch over all layers.
+// of the stream has completed).  Sized for a launch over all layers.  It exists twice and
+// launches alternate between the two sets, so that a launch which does not wait for its
+// predecessor (see Params::defer) never shares scratch with it.
 struct ScratchOff { size_t logit, head_sum, unit_sum, part_o, part_ml, keys, list_a, list_b, end; };
 // A launch plan: the CTAs' start table and the work-sharing counters of the launches that use it.
 // There is one per layer (launches of that layer alone) and one more for launches over several
 // layers, sized for all of them.
 struct PlanOff {
     size_t cta_unit0, cta_head0, cta_headn, cta_t0, unit_next0, unit_chunk, tile_begin, unit_cta0, next, cnt,
-        launch_no, end;
+        launch_no, tq_ctrl, tq_items, fin, end;
 };
 struct Layout {
     int layers, units, cap, rowb, lstride;
-    size_t status, stage_q, stage_k, stage_v, stage_out, scratch0, state0, plans0, plan_bytes, total;
+    size_t status, stage_q, stage_k, stage_v, stage_out, scratch0, scratch_bytes, state0, plans0, plan_bytes, total;
     ScratchOff so;  // offsets relative to the scratch base
     StateOff st;    // offsets relative to the state base
     PlanOff po;     // a single layer's plan, offsets relative to the plan's base
@@ -65,6 +67,9 @@ PlanOff make_plan_off(size_t nu) {
     p.next = take(2 * nu * 4);      // two copies each, alternating from launch to launch
     p.cnt = take(2 * nu * 8);
     p.launch_no = take((size_t)kMaxCtas * 4);   // per CTA: launches since the plan was (re)built
+    p.tq_ctrl = take(2 * 8);
+    p.tq_items = take(2 * nu * 4);
+    p.fin = take(2 * 8);
     p.end = o;
     return p;
 }
@@ -104,7 +109,8 @@ bool make_layout(int layers, int batch, int q_heads, int kv_heads, int head_dim,
     L.so.list_a = take(UA * C * 4);
     L.so.list_b = take(UA * C * 4);
     L.so.end = o;
-    L.state0 = L.scratch0 + o;
+    L.scratch_bytes = o;
+    L.state0 = L.scratch0 + 2 * o;
     o = 0;
     auto arr = [&](size_t bytes_per_layer) { ArrOff a{o, bytes_per_layer}; o = align_up(o + bytes_per_layer * NL); return a; };
     L.st.Kp = arr(U * max_prefill * L.rowb);
@@ -168,10 +174,19 @@ __global__ void host_gather_kernel(const HostPiece a, const HostPiece b, const H
     if (i < c3.n16) c3.dst[i] = c3.src[i];
 }
 
-// Test hook of mkv_debug_withhold_tile: one tile of unit `u` counts as never delivered.
-__global__ void withhold_kernel(int2* cnt, int n_units, int u) {
-    cnt[u] = make_int2(-1, 0);
-    cnt[n_units + u] = make_int2(-1, 0);
+// Test hooks.  what = 0: one tile of unit `u` counts as never delivered (both copies of its count
+// start at -1), so its tail never becomes due.  what = 1: the queue of due tails claims to hold one
+// more entry than will ever be written, so a tail group that takes it waits for its content.
+__global__ void debug_kernel(LayerDev L, int u, int what) {
+    if (what == 0) {
+        L.cnt[u] = make_int2(-1, 0);
+        L.cnt[L.n_units + u] = make_int2(-1, 0);
+    } else {
+        L.tq_ctrl[0] = make_int2(0, 1);
+        L.tq_ctrl[1] = make_int2(0, 1);
+        L.tq_items[0] = 0;
+        L.tq_items[L.n_units] = 0;
+    }
 }
 
 // The device's view of pinned host memory [p, p + bytes), or nullptr if the GPU cannot read it
@@ -192,6 +207,7 @@ constexpr int kMinChunk = 2;   // tiles per pull of a unit's counter, lower boun
 
 struct StartTable {
     int n_ctas = 0;
+    long long tiles = 0;      // all units' tiles with full decode pools
     std::vector<int32_t> lp, next0, chunk, cta_unit0, cta_head0, cta_headn;
     // reproducible mode
     std::vector<int32_t> tile_begin, cta_t0, unit_cta0;
@@ -232,6 +248,7 @@ StartTable build_start_table(int units, int budget, const int32_t* unit_lens, in
     const long long home_cap = (long long)(kMaxHome - 1) * t_all / t_max;
     const int n_ctas = (int)std::max<long long>(1, std::min<long long>(std::min<long long>(n_ctas_max, t_all / 2), home_cap));
     T.n_ctas = n_ctas;
+    T.tiles = t_all;
     T.cta_unit0.assign(n_ctas, 0);
     T.cta_head0.assign(n_ctas, 0);
     T.cta_headn.assign(n_ctas, 0);
@@ -292,7 +309,11 @@ struct mkv_ctx {
     // per plan (layers single-layer plans, then the several-layer plan)
     std::vector<char> stepped;   // a launch has used the plan since it was (re)built
     std::vector<int> n_ctas;
+    std::vector<int> tiles_per_cta;   // per plan: a CTA's even share of the plan's tiles
     int stack_layer0, stack_n;   // layers the several-layer plan is built for (stack_n = 0: none)
+    // the previous kernel launch of the context: its layers, stream and set of scratch
+    int last_layer0, last_n, scratch_set;
+    void* last_stream;
     std::vector<std::vector<int32_t>> lens;   // per layer, per (sequence, KV head) unit
     int64_t launches;
     std::vector<PinEntry> pins;  // host buffers already looked up by mkv_decode_step_host
@@ -306,8 +327,8 @@ inline uint8_t* plan_base(const mkv_ctx* c, int plan) {
 inline const PlanOff& plan_off(const mkv_ctx* c, int plan) { return plan < c->layers ? c->lay.po : c->lay.pso; }
 
 // Device view of layers [layer0, layer0 + n) as one list of n * units units, with launch plan `plan`.
-LayerDev layer_dev(const mkv_ctx* c, int layer0, int n, int plan) {
-    uint8_t* sb = c->ws + c->lay.scratch0;
+LayerDev layer_dev(const mkv_ctx* c, int layer0, int n, int plan, int set = 0) {
+    uint8_t* sb = c->ws + c->lay.scratch0 + c->lay.scratch_bytes * (size_t)set;
     uint8_t* stb = c->ws + c->lay.state0;
     uint8_t* pb = plan_base(c, plan);
     const StateOff& o = c->lay.st;
@@ -342,6 +363,9 @@ LayerDev layer_dev(const mkv_ctx* c, int layer0, int n, int plan) {
     d.next = (int32_t*)(pb + po.next);
     d.cnt = (int2*)(pb + po.cnt);
     d.launch_no = (uint32_t*)(pb + po.launch_no);
+    d.tq_ctrl = (int2*)(pb + po.tq_ctrl);
+    d.tq_items = (int32_t*)(pb + po.tq_items);
+    d.fin = (int2*)(pb + po.fin);
     d.part_o = (float*)(sb + so.part_o);
     d.part_ml = (float*)(sb + so.part_ml);
     d.unit_step = (int32_t*)at(o.unit_step);
@@ -356,7 +380,8 @@ LayerDev layer_dev(const mkv_ctx* c, int layer) { return layer_dev(c, layer, 1, 
 Params make_params(const mkv_ctx* c, int layer0, int n, int plan, const void* q, const void* k_new,
                    const void* v_new, void* out, int mode) {
     Params p;
-    p.L = layer_dev(c, layer0, n, plan);
+    p.L = layer_dev(c, layer0, n, plan, c->scratch_set ^ 1);   // the set the previous launch did not use
+    p.defer = 0;
     p.q = q; p.k_new = k_new; p.v_new = v_new; p.out = out;
     p.status = (int32_t*)(c->ws + c->lay.status);
     p.batch = c->batch * n; p.q_heads = c->q_heads; p.kv_heads = c->kv_heads; p.group = c->group;
@@ -376,15 +401,23 @@ Params make_params(const mkv_ctx* c, int layer0, int n, int plan, const void* q,
     return p;
 }
 
-mkv_status launch_step(mkv_ctx* c, int plan, const Params& p, cudaStream_t st) {
+mkv_status launch_step(mkv_ctx* c, int plan, int layer0, int n, Params p, cudaStream_t st, bool staged_inputs = false) {
     // The first launch after a plan was (re)built must see the prefill's copies complete before
     // it reads the table and the pool; later ones may overlap their start with the previous
     // kernel's end.
     const bool overlap = c->pdl && c->stepped[plan];
+    // A launch whose layers are all different from those of the context's previous launch on the
+    // same stream has nothing in common with it (its own pools, scores and counters; the other
+    // set of scratch), and with the caller's inputs final it need not wait for it at all.
+    const bool disjoint = c->last_n > 0 && (layer0 >= c->last_layer0 + c->last_n || c->last_layer0 >= layer0 + n);
+    p.defer = (overlap && c->use_mma && p.early_inputs && !staged_inputs && disjoint && c->last_stream == (void*)st) ? 1 : 0;
+    p.trigger_after = std::max(1, c->tiles_per_cta[plan] / 2);
     cudaError_t e = c->use_mma ? launch_mma(p, st, overlap, c->stages) : launch_simt(p, c->kv_dtype, st);
     if (e != cudaSuccess) return MKV_ERR_CUDA;
     c->launches += 1;
     c->stepped[plan] = 1;
+    c->last_layer0 = layer0; c->last_n = n; c->last_stream = (void*)st;
+    c->scratch_set ^= 1;
     return MKV_OK;
 }
 
@@ -417,6 +450,7 @@ mkv_status upload_plan(mkv_ctx* c, int plan, int units, const int32_t* unit_lens
     const StartTable T = build_start_table(units, c->budget_max, unit_lens, c->n_ctas_max, c->head_tiles,
                                            (c->flags & MKV_FLAG_REPRODUCIBLE) != 0);
     c->n_ctas[plan] = T.n_ctas;
+    c->tiles_per_cta[plan] = (int)std::max<long long>(1, T.tiles / T.n_ctas);
     uint8_t* pb = plan_base(c, plan);
     const PlanOff& po = plan_off(c, plan);
     const size_t U = (size_t)units, N = (size_t)T.n_ctas;
@@ -436,6 +470,7 @@ mkv_status upload_plan(mkv_ctx* c, int plan, int units, const int32_t* unit_lens
     up(po.next + U * 4, T.next0, U);
     ok &= cudaMemsetAsync(pb + po.cnt, 0, 2 * U * 8, st) == cudaSuccess;
     ok &= cudaMemsetAsync(pb + po.launch_no, 0, (size_t)kMaxCtas * 4, st) == cudaSuccess;
+    ok &= cudaMemsetAsync(pb + po.tq_ctrl, 0, po.end - po.tq_ctrl, st) == cudaSuccess;   // queue, entries, finish counts
     // (the host vectors are pageable: the runtime has staged them before each call returns)
     c->stepped[plan] = 0;
     return ok ? MKV_OK : MKV_ERR_CUDA;
@@ -577,7 +612,9 @@ mkv_status mkv_create(int layers, int q_heads, int kv_heads, int head_dim, int b
     c->prefilled.assign(layers, 0);
     c->stepped.assign(layers + 1, 0);
     c->n_ctas.assign(layers + 1, 0);
+    c->tiles_per_cta.assign(layers + 1, 1);
     c->stack_layer0 = 0; c->stack_n = 0;
+    c->last_layer0 = 0; c->last_n = 0; c->scratch_set = 0; c->last_stream = nullptr;
     c->lens.assign(layers, std::vector<int32_t>((size_t)batch * kv_heads, 0));
     c->launches = 0;
     *out_ctx = c;
@@ -665,8 +702,9 @@ mkv_status mkv_prefill_units(mkv_ctx* c, int layer, const void* K, const void* V
     ok &= cudaMemsetAsync(d.unit_step, 0, U * 4, st) == cudaSuccess;
     ok &= cudaMemsetAsync(d.seq_ticket, 0, (size_t)c->batch * 4, st) == cudaSuccess;
     // the rows of head sums are zero between steps; a step that was cut short may have left some
-    ok &= cudaMemsetAsync(c->ws + L.scratch0 + L.so.head_sum, 0,
-                          (size_t)L.layers * c->batch * L.lstride * 4, st) == cudaSuccess;
+    for (int set = 0; set < 2; ++set)
+        ok &= cudaMemsetAsync(c->ws + L.scratch0 + L.scratch_bytes * set + L.so.head_sum, 0,
+                              (size_t)L.layers * c->batch * L.lstride * 4, st) == cudaSuccess;
     if (!ok) return MKV_ERR_CUDA;
     if (maxlen > 0) {
         const long long total = (long long)U * src_rows * (L.rowb / 16);
@@ -689,7 +727,7 @@ mkv_status mkv_decode_step(mkv_ctx* c, int layer, const void* q, const void* k_n
     DeviceGuard guard(c->device);
     if (!guard.ok) return MKV_ERR_CUDA;
     const Params p = make_params(c, layer, 1, layer, q, k_new, v_new, out, kModeDecode);
-    return launch_step(c, layer, p, (cudaStream_t)stream);
+    return launch_step(c, layer, layer, 1, p, (cudaStream_t)stream);
 }
 
 mkv_status mkv_decode_step_layers(mkv_ctx* c, int layer0, int n_layers, const void* q, const void* k_new,
@@ -702,7 +740,7 @@ mkv_status mkv_decode_step_layers(mkv_ctx* c, int layer0, int n_layers, const vo
     if (!guard.ok) return MKV_ERR_CUDA;
     if ((s = ensure_stack_plan(c, layer0, n_layers, (cudaStream_t)stream)) != MKV_OK) return s;
     const Params p = make_params(c, layer0, n_layers, c->layers, q, k_new, v_new, out, kModeDecode);
-    return launch_step(c, c->layers, p, (cudaStream_t)stream);
+    return launch_step(c, c->layers, layer0, n_layers, p, (cudaStream_t)stream);
 }
 
 mkv_status mkv_attend_only_layers(mkv_ctx* c, int layer0, int n_layers, const void* q, void* out, void* stream) {
@@ -714,7 +752,7 @@ mkv_status mkv_attend_only_layers(mkv_ctx* c, int layer0, int n_layers, const vo
     if (!guard.ok) return MKV_ERR_CUDA;
     if ((s = ensure_stack_plan(c, layer0, n_layers, (cudaStream_t)stream)) != MKV_OK) return s;
     const Params p = make_params(c, layer0, n_layers, c->layers, q, nullptr, nullptr, out, kModeAttendOnly);
-    return launch_step(c, c->layers, p, (cudaStream_t)stream);
+    return launch_step(c, c->layers, layer0, n_layers, p, (cudaStream_t)stream);
 }
 
 mkv_status mkv_decode_step_host(mkv_ctx* c, int layer, const void* qh, const void* kh, const void* vh, void* outh,
@@ -781,7 +819,7 @@ mkv_status mkv_decode_step_host(mkv_ctx* c, int layer, const void* qh, const voi
     void* const kernel_out = direct ? direct : (void*)dout;
     Params p = make_params(c, layer, 1, layer, dq, dk, dv, kernel_out, kModeDecode);
     p.early_inputs = 0;   // the inputs arrive through the staging area, written by the kernel or copy just ahead
-    const mkv_status s = launch_step(c, layer, p, st);
+    const mkv_status s = launch_step(c, layer, layer, 1, p, st, true);
     if (s != MKV_OK) return s;
     if (!direct && cudaMemcpyAsync(outh, dout, nq * os, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return MKV_ERR_CUDA;
@@ -795,7 +833,7 @@ mkv_status mkv_attend_only(mkv_ctx* c, int layer, const void* q, void* out, void
     DeviceGuard guard(c->device);
     if (!guard.ok) return MKV_ERR_CUDA;
     const Params p = make_params(c, layer, 1, layer, q, nullptr, nullptr, out, kModeAttendOnly);
-    return launch_step(c, layer, p, (cudaStream_t)stream);
+    return launch_step(c, layer, layer, 1, p, (cudaStream_t)stream);
 }
 
 mkv_status mkv_set_budget(mkv_ctx* c, int budget) {
@@ -836,14 +874,15 @@ mkv_status mkv_get_grid(const mkv_ctx* c, int layer, int32_t* n_ctas, int32_t* n
     return MKV_OK;
 }
 
-mkv_status mkv_debug_withhold_tile(mkv_ctx* c, int layer, int b, int g) {
+mkv_status mkv_debug_inject(mkv_ctx* c, int layer, int what, int b, int g) {
     if (!layer_ok(c, layer) || b < 0 || b >= c->batch || g < 0 || g >= c->kv_heads) return MKV_ERR_INVALID_ARG;
+    if (what != MKV_INJECT_LOST_TILE && what != MKV_INJECT_EMPTY_QUEUE_ENTRY) return MKV_ERR_INVALID_ARG;
     if (!c->prefilled[layer]) return MKV_ERR_BAD_STATE;
     if (!c->use_mma) return MKV_ERR_UNSUPPORTED;
     DeviceGuard guard(c->device);
     if (!guard.ok || cudaDeviceSynchronize() != cudaSuccess) return MKV_ERR_CUDA;
     const LayerDev d = layer_dev(c, layer);
-    withhold_kernel<<<1, 1>>>(d.cnt, d.n_units, b * c->kv_heads + g);
+    debug_kernel<<<1, 1>>>(d, b * c->kv_heads + g, what == MKV_INJECT_LOST_TILE ? 0 : 1);
     if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return MKV_ERR_CUDA;
     return MKV_OK;
 }

@@ -29,9 +29,12 @@
 //     ring stage borrowed from the producer and go straight on to the next unit; the merge
 //     warp folds the four states into one partial in global memory, returns the stage, adds
 //     the visit's tiles to the unit's count.
-//   * four TAIL warps, which watch the counts of the units assigned to this CTA and run a
-//     unit's tail (fresh token, combine, probabilities, momentum update, selection,
-//     append/compaction) as soon as its count is complete, while the stream continues.
+//   * four TAIL warps, which run a unit's tail (fresh token, combine, probabilities, momentum
+//     update, selection, append/compaction) while the stream continues.  The merge warp whose
+//     delivery completes a unit hands it to its own CTA's tail warps (a word in shared memory);
+//     if they are busy the unit goes into a queue in global memory that every idle tail group
+//     looks at.  A CTA therefore leaves as soon as its own streaming is over and it has no
+//     tail in hand: it never waits for a unit that other CTAs are still working on.
 // Every wait is bounded (the context's wait limit): on expiry the kernel records
 // MKV_ERR_TIMEOUT, every role drains (the producer waits, bounded again, for its copies in
 // flight) and the CTA returns.
@@ -43,6 +46,13 @@
 //   * early inputs: the caller's q is final when the launch is enqueued, so the consumers may
 //     work through the CTA's reserved prompt tiles (frozen rows) while the previous kernel of
 //     the stream is still running its last tails; everything else waits for it as usual.
+//     When, on top of that, the previous kernel worked on other layers (the host knows), the
+//     launch shares nothing with it -- layers are independent instances of Algorithm 1 and the
+//     step scratch exists twice -- and is "deferred": no role waits at the start, CTAs stream as
+//     soon as they get an SM, and the producer passes the dependency wait about half-way through
+//     its share of the tiles, long after the previous kernel has ended.  Only then does the CTA
+//     allow the next launch to begin (whose CTAs take the SMs of this launch's CTAs as they
+//     finish), so at most two launches are ever in flight and they complete in order.
 //   * reproducible mode: no counters; every CTA covers a fixed range of the global tile
 //     sequence and delivers a fixed partial slot, so the same inputs give the same bits.
 #include "mkv_launch.h"
@@ -96,9 +106,12 @@ struct Control {
     StageMeta meta[kMaxStages];
     ExchangeRef xq[kMaxStages];
     int abort_flag;
-    int tail_unit;     // partial slots of the unit whose tail is due, or -1
+    int tail_unit;     // the unit whose tail the group runs next, or -1: leave
     int par;           // parity of this launch (the producer finds it after the dependency wait); -1 before
+    int mail;          // unit handed to this CTA's tail warps by its merge warp; kMailEmpty / kMailBusy otherwise
+    int stream_done;   // the merge warp has delivered this CTA's last visit
 };
+enum : int { kMailEmpty = -1, kMailBusy = -2 };
 
 constexpr size_t smem_bytes(int nst) {
     return (size_t)nst * kStageBytes + kQSlots * kQSlotBytes + sizeof(TailSmem<kTailThreads>) + sizeof(Control) + 64;
@@ -124,49 +137,104 @@ __device__ inline bool wait_or_abort(uint32_t bar, uint32_t parity, Control* ctl
     }
 }
 
-// The tail warps' loop over the units this CTA looks after.  While a unit is still being
-// streamed the group already fetches what its tail needs and the step does not change
-// (tail_prefetch); thread 0 then watches the unit's counters, which arrive as one 8-byte
-// word (tiles delivered, partial slots taken).
+// Takes one entry of the queue of due tails, if there is one: the unit, -1 (nothing queued) or
+// -2 (the entry was never written within the wait limit).
+__device__ inline int queue_take(const Params& p, Control* ctl, int par) {
+    const LayerDev& L = p.L;
+    int2* ctrl = L.tq_ctrl + par;
+    for (;;) {
+        const unsigned long long w = *reinterpret_cast<const volatile unsigned long long*>(ctrl);
+        const int taken = (int)(unsigned)(w & 0xffffffffull), put = (int)(unsigned)(w >> 32);
+        if (taken >= put) return -1;
+        if (atomicCAS(&ctrl->x, taken, taken + 1) != taken) continue;      // another group was faster
+        // the entry is written right after its number was drawn: a short, bounded wait
+        const volatile int32_t* item = L.tq_items + (size_t)par * L.n_units + min(taken, L.n_units - 1);
+        const unsigned long long t0 = ptx::globaltimer_ns();
+        for (;;) {
+            const int v = *item;
+            if (v > 0) return v - 1;
+            if (aborted(ctl)) return -2;
+            if (ptx::globaltimer_ns() - t0 > p.wait_ns) { note_timeout(p, ctl); return -2; }
+        }
+    }
+}
+
+// Puts a completed unit into the queue (merge warp, one lane).
+__device__ inline void queue_put(const LayerDev& L, int par, int u) {
+    const int idx = atomicAdd(&L.tq_ctrl[par].y, 1);
+    *reinterpret_cast<volatile int32_t*>(L.tq_items + (size_t)par * L.n_units + min(idx, L.n_units - 1)) = u + 1;
+}
+
+// The tail warps' loop.  Thread 0 looks for work: first the word its own merge warp writes, then
+// the queue; when the CTA's streaming is over and neither holds anything the group leaves.
 // LAYER: the tails of a sequence's KV heads score together (Eq. 4 over all heads of the layer).
 template <int GB, bool LAYER>
 __device__ void tail_group(const Params& p, Control* ctl, TailSmem<kTailThreads>* tsm, int tt) {
     const LayerDev& L = p.L;
-    const bool dec = (p.mode == kModeDecode);
-    for (int u = blockIdx.x; u < L.n_units; u += gridDim.x) {
-        TailPre<kTailThreads, GB> pre;
-        tail_prefetch<__nv_bfloat16, kTailThreads, GB, LAYER>(p, u, *tsm, tt, pre);
+    int par = -1;                  // (thread 0)
+    for (;;) {
         if (tt == 0) {
-            const int total = p.det ? L.tile_begin[u + 1] - L.tile_begin[u]
-                                    : unit_tiles(L.unit_lp[u], min(pre.n_dec, p.cap - (dec ? 1 : 0)));
+            int unit = -1;
             const unsigned long long t0 = ptx::globaltimer_ns();
-            int slots = -1;
-            int par = tsm->par;
-            while (par < 0) {   // first unit: the producer has not read the launch's parity yet
-                par = *reinterpret_cast<const volatile int*>(&ctl->par);
-                if (par >= 0) { tsm->par = par; break; }
+            for (unsigned spin = 0;; ++spin) {
+                if (par < 0) {     // the producer has not read the launch's parity yet
+                    par = *reinterpret_cast<const volatile int*>(&ctl->par);
+                    if (par >= 0) tsm->par = par;
+                }
+                const int done = *reinterpret_cast<const volatile int*>(&ctl->stream_done);
+                const int m = *reinterpret_cast<const volatile int*>(&ctl->mail);
+                if (m >= 0) {      // handed over by this CTA's merge warp
+                    unit = m;
+                    *reinterpret_cast<volatile int*>(&ctl->mail) = kMailBusy;
+                    break;
+                }
+                // the queue: at once when this CTA has nothing else to do, now and then otherwise
+                if (par >= 0 && (done || (spin & 7u) == 0u)) {
+                    const int q = queue_take(p, ctl, par);
+                    if (q >= 0) {
+                        unit = q;
+                        atomicCAS(&ctl->mail, (int)kMailEmpty, (int)kMailBusy);   // (a unit posted meanwhile stays posted)
+                        break;
+                    }
+                    if (q == -2) break;
+                }
+                if (done) {        // `done` was read before the word and the queue: nothing can follow
+                    if (*reinterpret_cast<const volatile int*>(&ctl->mail) >= 0) continue;
+                    break;
+                }
                 if (aborted(ctl)) break;
                 if (ptx::globaltimer_ns() - t0 > p.wait_ns) { note_timeout(p, ctl); break; }
+                __nanosleep(64);
             }
-            const int2* cnt_u = L.cnt + (size_t)max(par, 0) * L.n_units + u;
-            for (; par >= 0;) {
-                const unsigned long long w = *reinterpret_cast<const volatile unsigned long long*>(cnt_u);
-                if ((int)(unsigned)(w & 0xffffffffull) >= total) { slots = (int)(unsigned)(w >> 32); break; }
-                if (aborted(ctl)) break;
-                if (ptx::globaltimer_ns() - t0 > p.wait_ns) { note_timeout(p, ctl); break; }
-                __nanosleep(100);
-            }
-            ctl->tail_unit = slots;
+            ctl->tail_unit = unit;
         }
         bar_sync(1, kTailThreads);
-        const int slots = ctl->tail_unit;
+        const int u = ctl->tail_unit;
         bar_sync(1, kTailThreads);     // everyone has read it before thread 0 writes again
-        if (slots < 0) break;
+        if (u < 0) break;
         __threadfence();
         if (tt == 0) MKV_TR_ADD(6, 1);
+        const int slots = __ldcg(&L.cnt[(size_t)tsm->par * L.n_units + u].y);
+        TailPre<kTailThreads, GB> pre;
+        tail_prefetch<__nv_bfloat16, kTailThreads, GB, LAYER>(p, u, *tsm, tt, pre);
         if constexpr (LAYER) layer_unit_tail<__nv_bfloat16, kTailThreads, 1, GB>(p, u, slots, pre, *tsm, tt);
         else unit_tail<__nv_bfloat16, kTailThreads, 1, GB>(p, u, slots, pre, *tsm, tt);
-        if (tt == 0) MKV_TR(5);
+        bar_sync(1, kTailThreads);     // the whole group is through with the unit
+        if (tt == 0) {
+            MKV_TR(5);
+            __threadfence();
+            atomicAdd(&L.fin[tsm->par].x, 1);
+            atomicCAS(&ctl->mail, (int)kMailBusy, (int)kMailEmpty);
+        }
+    }
+    // Leaving.  The last CTA of the launch to get here checks that every unit had its tail (they
+    // all have unless a tile was never delivered).
+    if (tt == 0 && tsm->par >= 0) {
+        __threadfence();
+        int2* fin = L.fin + tsm->par;
+        if (atomicAdd(&fin->y, 1) == (int)gridDim.x - 1) {
+            if (__ldcg(&fin->x) != L.n_units && !aborted(ctl)) atomicCAS(p.status, kStatusOk, kStatusDeviceCheck);
+        }
     }
 }
 
@@ -197,14 +265,18 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         ctl->abort_flag = 0;
         ctl->tail_unit = -1;
         ctl->par = -1;
+        ctl->mail = kMailEmpty;
+        ctl->stream_done = 0;
         tsm->par = -1;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async();
     }
     __syncthreads();
     if (tid == 0) { MKV_TR(0); MKV_TR_SET(6, 0); }
-    // The next kernel of the stream may start as soon as SMs free up; it does its own waiting.
-    ptx::griddep_launch_dependents();
+    const bool defer = p.defer != 0;
+    // The next kernel of the stream may begin once every CTA of this one has said so
+    // (griddepcontrol.launch_dependents) -- which a CTA does only after it has itself passed the
+    // dependency wait: when the next kernel runs, everything before this one is complete.
 
     if (warp == kProducerWarp) {
         // ================================ producer =====================================
@@ -214,6 +286,8 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         uint32_t issued = 0;       // bit s: a copy into stage s may still be in flight
         uint32_t issued_par = 0;   // parity its full barrier completes with
         bool ok = true;
+        int issued_all = 0;        // tiles issued by this CTA (lane 0)
+        bool let_in = !defer;      // the next launch may begin as far as this CTA is concerned (lane 0)
         // K and V are read exactly once per step: let them leave L2 first, so that the
         // step's scratch (logits, partials) and the scores stay resident for the tails
         const unsigned long long stream_policy = ptx::l2_policy_evict_first();
@@ -244,6 +318,14 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             issued |= 1u << stage;
             issued_par = (issued_par & ~(1u << stage)) | (phase << stage);
             advance();
+            if (!let_in && ++issued_all >= p.trigger_after) {
+                // deferred launch, half-way: the previous kernel ended long ago, so the wait
+                // returns at once; it orders this launch's end behind that kernel's
+                ptx::griddep_wait();
+                ptx::griddep_launch_dependents();
+                let_in = true;
+                if (defer) MKV_TR(7);
+            }
             return true;
         };
         // the unit's G query rows, one padded row each, into the next query slot
@@ -295,8 +377,11 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
                 if (ok) { if (sent == 0) MKV_TR(1); ++sent; ++mine; }
             }
         }
-        ptx::griddep_wait();
-        if (lane == 0) MKV_TR(7);
+        if (!defer) {
+            ptx::griddep_wait();
+            ptx::griddep_launch_dependents();
+        }
+        if (lane == 0 && !defer) MKV_TR(7);
         // Loads first, then the query copy, then their use: the consumers wait for the query, which
         // must not wait for a load's round trip.
         int n_old = L.n_dec[u];
@@ -316,6 +401,15 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             *reinterpret_cast<volatile int*>(&ctl->par) = par;
         }
         par = __shfl_sync(0xffffffffu, par, 0);
+        if (blockIdx.x == 0) {
+            // The other copy of the queue and of the finish counts was used by this layer's
+            // previous launch, which is complete: empty it for the next one.
+            const int idle = par ^ 1;
+            const int used = min(__ldcg(&L.tq_ctrl[idle].y), L.n_units);
+            for (int i = lane; i < used; i += 32) L.tq_items[(size_t)idle * L.n_units + i] = 0;
+            __syncwarp();
+            if (lane == 0) { L.tq_ctrl[idle] = make_int2(0, 0); L.fin[idle] = make_int2(0, 0); }
+        }
         int32_t* const nxt = L.next + (size_t)par * L.n_units;
         int2* const cnt = L.cnt + (size_t)par * L.n_units;
         int total = unit_tiles(lp, n_old);
@@ -422,6 +516,12 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             total = unit_tiles(lp, n_old);
             if (lane == 0) g = atomicAdd(&nxt[u], chunk);
         }
+        if (lane == 0 && !let_in) {
+            // a deferred launch's CTA that issued few tiles: streaming is over, same duty now
+            ptx::griddep_wait();
+            ptx::griddep_launch_dependents();
+            MKV_TR(7);
+        }
         if (lane == 0) {
             if (ok && acquire()) {
                 ctl->meta[stage].kind = kEntryEnd;
@@ -461,7 +561,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
                 break;
             }
             const StageMeta mt = ctl->meta[stage];
-            if (!waited && !mt.pre) { ptx::griddep_wait(); waited = true; }
+            if (!waited && !mt.pre && !defer) { ptx::griddep_wait(); waited = true; }
             if (warp == 0 && lane == 0 && xcount == 0 && mt.first) MKV_TR(2);
             if (mt.kind == kEntryEnd) {
                 if (warp == 0 && lane == 0) MKV_TR(3);
@@ -603,7 +703,7 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
         // Folds the four consumer states of a unit visit into one partial in global memory,
         // gives the borrowed stage back, adds the visit's tiles to the unit's count and, when
         // that completes the unit, publishes the unit in the layer's queue of due tails.
-        ptx::griddep_wait();
+        if (!defer) ptx::griddep_wait();
         for (int x = 0;; ++x) {
             const int xs = x % nst;
             if (!wait_or_abort(ptx::smem_u32(&ctl->xfull[xs]), (uint32_t)((x / nst) & 1), ctl, p.wait_ns)) {
@@ -647,22 +747,23 @@ __global__ void __launch_bounds__(kThreads, 2) mma_kernel(const Params p, const 
             if (lane < kConsumerWarps) ptx::mbar_arrive(ptx::smem_u32(&ctl->empty[ref.stage]));
             __threadfence();
             __syncwarp();
-            // The tail group that looks after this unit watches the count; nothing to announce.
             if (lane == 0) {
                 MKV_TR(4);
                 // (the producer wrote the parity before it sent this visit's first counter pull)
                 const int par = *reinterpret_cast<const volatile int*>(&ctl->par);
-                atomicAdd(&L.cnt[(size_t)par * L.n_units + u].x, ref.ntiles);
+                const int before = atomicAdd(&L.cnt[(size_t)par * L.n_units + u].x, ref.ntiles);
+                if (before + ref.ntiles == ref.total) {
+                    // the unit is complete: its tail goes to this CTA's tail warps, or, if they
+                    // have one in hand, to whichever group is idle
+                    if (atomicCAS(&ctl->mail, (int)kMailEmpty, u) != kMailEmpty) queue_put(L, par, u);
+                }
             }
         }
+        __syncwarp();
+        if (lane == 0) { __threadfence_block(); *reinterpret_cast<volatile int*>(&ctl->stream_done) = 1; }
     } else {
         // ================================ tail warps ===================================
-        // Unit tails are spread statically: this CTA's tail group looks after units
-        // blockIdx.x, blockIdx.x + gridDim.x, ...  It watches the unit's count of delivered
-        // tiles and runs the tail the moment the count is complete, so no CTA ever has two
-        // tails due at once (as long as there are at least as many CTAs as units) and nothing
-        // has to be announced or claimed.
-        ptx::griddep_wait();
+        if (!defer) ptx::griddep_wait();
         if (G <= 4) tail_group<4, LAYER>(p, ctl, tsm, tid - kTailTid0);
         else tail_group<8, LAYER>(p, ctl, tsm, tid - kTailTid0);
     }

@@ -14,6 +14,7 @@ MKV_SCORE_GROUP_MEAN, MKV_SCORE_LAYER_MEAN = 0, 1
 MKV_KERNEL_AUTO, MKV_KERNEL_SIMT, MKV_KERNEL_MMA = 0, 1, 2
 MKV_FLAG_RECORD_PROBS, MKV_FLAG_INPUTS_READY, MKV_FLAG_REPRODUCIBLE = 1, 2, 4
 MKV_OPT_RING_STAGES, MKV_OPT_HEAD_TILES, MKV_OPT_WAIT_LIMIT_US, MKV_OPT_OVERLAP = 1, 2, 3, 4
+MKV_INJECT_LOST_TILE, MKV_INJECT_EMPTY_QUEUE_ENTRY = 0, 1
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmkv.so")
@@ -24,7 +25,7 @@ EXPORTED_SYMBOLS = [
     "mkv_status_sync", "mkv_launch_count", "mkv_get_decode_state", "mkv_get_last_evicted",
     "mkv_get_last_probs", "mkv_read_kv", "mkv_get_step", "mkv_status_string", "mkv_attend_noalloc", "mkv_plan_starts", "mkv_prefill_units",
     "mkv_recency_diagnostics", "mkv_set_option", "mkv_plan_ranges", "mkv_grid_limit", "mkv_decode_step_layers",
-    "mkv_attend_only_layers", "mkv_get_grid", "mkv_debug_withhold_tile",
+    "mkv_attend_only_layers", "mkv_get_grid", "mkv_debug_inject",
 ]
 
 
@@ -80,7 +81,7 @@ def load_library(path: str | None = None):
     L.mkv_decode_step_layers.argtypes = [vp, C.c_int, C.c_int, vp, vp, vp, vp, vp]
     L.mkv_attend_only_layers.argtypes = [vp, C.c_int, C.c_int, vp, vp, vp]
     L.mkv_get_grid.argtypes = [vp, C.c_int, i32p, i32p]
-    L.mkv_debug_withhold_tile.argtypes = [vp, C.c_int, C.c_int, C.c_int]
+    L.mkv_debug_inject.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int]
     L.mkv_status_string.restype = C.c_char_p
     L.mkv_status_string.argtypes = [C.c_int]
     if path is None:
@@ -271,8 +272,8 @@ class MomentKV:
         _check(self._L.mkv_get_grid(self._ctx, layer, C.byref(n), C.byref(nmax)), "mkv_get_grid")
         return int(n.value), int(nmax.value)
 
-    def debug_withhold_tile(self, layer, b, g):
-        _check(self._L.mkv_debug_withhold_tile(self._ctx, layer, b, g), "mkv_debug_withhold_tile")
+    def debug_inject(self, layer, what, b=0, g=0):
+        _check(self._L.mkv_debug_inject(self._ctx, layer, what, b, g), "mkv_debug_inject")
 
     def set_budget(self, budget):
         _check(self._L.mkv_set_budget(self._ctx, int(budget)), "mkv_set_budget")

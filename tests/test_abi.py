@@ -161,6 +161,6 @@ def test_new_calls_check_their_arguments(lib):
     assert lib.mkv_set_option(None, 1, 3) == 1
     assert lib.mkv_decode_step_layers(None, 0, 1, one, one, one, one, None) == 1
     assert lib.mkv_attend_only_layers(None, 0, 1, one, one, None) == 1
-    assert lib.mkv_debug_withhold_tile(None, 0, 0, 0) == 1
+    assert lib.mkv_debug_inject(None, 0, 0, 0, 0) == 1
     n, m = C.c_int32(0), C.c_int32(0)
     assert lib.mkv_get_grid(None, 0, C.byref(n), C.byref(m)) == 1

@@ -215,6 +215,54 @@ def test_early_inputs_overlap_keeps_parity(mode, head_tiles):
     ctx.close()
 
 
+@pytest.mark.parametrize("mode", ["group", "layer"])
+@pytest.mark.parametrize("n_layers", [2, 3])
+def test_steps_of_different_layers_run_side_by_side(mode, n_layers):
+    """With MKV_FLAG_INPUTS_READY a step on another layer than the previous one does not wait for
+    it: it streams alongside (its own pools and counters, the other set of scratch) and only
+    completes behind it.  Layers are cycled back to back, many steps per synchronisation, each
+    step with an output buffer of its own; every output and, after every burst, every pool and
+    score is compared with the per-layer oracles.  With two layers a step's successor-but-one is
+    the same layer again, which must see the step complete."""
+    import torch
+    w = CONFIGS["llama_b16"].with_(batch=5, prefill=(300, 2500), steps=120, budget=64, variant="hot", n_heavy=3)
+    smode, omode = ((mkv.MKV_SCORE_LAYER_MEAN, O.LAYER_MEAN) if mode == "layer" else (mkv.MKV_SCORE_GROUP_MEAN, O.GROUP_MEAN))
+    ws = [w.with_(seed=50 + l) for l in range(n_layers)]
+    max_pre = max(int(x.prefill_lens().max()) for x in ws)
+    ctx = mkv.MomentKV(n_layers, w.q_heads, w.kv_heads, w.head_dim, w.budget, w.beta, w.batch, max_pre, out_dtype=mkv.MKV_F32,
+                       score_mode=smode, flags=mkv.MKV_FLAG_INPUTS_READY)
+    streams = [BatchStream(ws[l], l) for l in range(n_layers)]
+    oracles = [prefill_both(ctx, ws[l], streams[l], layer=l, mode=omode)[0] for l in range(n_layers)]
+    dt, dev = ctx.torch_kv_dtype(), ctx.device
+    burst = 20
+    outs = torch.zeros((burst, n_layers, w.batch, w.q_heads, w.head_dim), dtype=torch.float32, device=dev)
+    for start in range(0, w.steps, burst):
+        (qs, ks, vs), (qd, kd, vd) = stacked_inputs(streams, burst, torch, dt, dev)
+        torch.cuda.synchronize()                          # the inputs are final before any step is enqueued
+        for j in range(burst):
+            for l in range(n_layers):
+                ctx.decode_step(l, qd[j, l], kd[j, l], vd[j, l], outs[j, l])
+        ctx.status_sync()
+        got = outs.double().cpu().numpy()
+        for j in range(burst):
+            for l in range(n_layers):
+                for b in range(w.batch):
+                    ref = oracles[l][b].attend_update(qs[j, l, b], ks[j, l, b], vs[j, l, b])
+                    rowmax = np.abs(ref).max(axis=1)
+                    assert (np.abs(got[j, l, b] - ref).max(axis=1) <= 2e-3 * rowmax).all(), (start + j, l, b)
+                    oracles[l][b].evict()
+        for l in range(n_layers):
+            for b in range(w.batch):
+                for g in range(w.kv_heads):
+                    pos, sc = ctx.decode_state(l, b, g)
+                    o_pos, o_sc, _ = oracles[l][b].decode_state(g)
+                    np.testing.assert_array_equal(np.sort(pos), np.sort(o_pos))
+                    np.testing.assert_allclose(sc[np.argsort(pos)], o_sc[np.argsort(o_pos)], rtol=1e-4)
+    for l in range(n_layers):
+        assert ctx.step_count(l) == w.steps
+    ctx.close()
+
+
 @pytest.mark.parametrize("case", ["mma_group", "mma_layer", "simt_f32", "simt_f32_layer"])
 def test_reproducible_mode_gives_the_same_bits_twice(case):
     """MKV_FLAG_REPRODUCIBLE: two contexts fed the same 300 steps (ragged batch, evictions of all
@@ -291,12 +339,16 @@ def test_ring_depth_resizes_the_grid(stages):
     assert rep.max_out_err <= 2e-3 and rep.max_score_err <= 1e-4
 
 
-def test_a_wait_that_runs_out_ends_the_step_with_a_status():
-    """The error path of the kernel's bounded waits, made to happen from the host: one tile of one
-    unit is marked as never delivered, so that unit's finishing part waits for a count that cannot
-    come, gives up at the wait limit (set to 20 ms here) and the step ends with MKV_ERR_TIMEOUT in
-    the sticky status.  Nothing traps and nothing spins without bound.  After mkv_reset and a new
-    prefill the context passes a parity run again."""
+@pytest.mark.parametrize("what", ["empty_queue_entry", "lost_tile"])
+def test_injected_errors_end_the_step_with_a_status(what):
+    """The error paths of the tensor-core kernel, made to happen from the host.
+    empty_queue_entry: the queue through which finished units reach idle CTAs claims an entry that
+    is never written; a CTA takes it, waits for its content, gives up at the wait limit (set to
+    20 ms here) and the step ends with MKV_ERR_TIMEOUT in the sticky status -- a bounded wait that
+    really runs out.  lost_tile: a tile of one unit counts as never delivered; the last CTA to
+    leave notices that a unit never had its finishing part: MKV_ERR_DEVICE_CHECK, without any
+    waiting.  Nothing traps and nothing spins without bound.  After mkv_reset and a new prefill
+    the context passes a parity run again."""
     import time
     import torch
     w = CONFIGS["llama_b1"].with_(batch=2, prefill=(100, 260), steps=60, budget=30, variant="hot", n_heavy=2)
@@ -306,7 +358,10 @@ def test_a_wait_that_runs_out_ends_the_step_with_a_status():
     oracles, _ = prefill_both(ctx, w, stream)
     rep = lockstep(ctx, w, stream, oracles, 20)
     assert rep.ok(), rep.failures[:5]
-    ctx.debug_withhold_tile(0, 1, 3)
+    if what == "lost_tile":
+        ctx.debug_inject(0, mkv.MKV_INJECT_LOST_TILE, 1, 3)
+    else:
+        ctx.debug_inject(0, mkv.MKV_INJECT_EMPTY_QUEUE_ENTRY)
     dt, dev = ctx.torch_kv_dtype(), ctx.device
     qs, ks, vs = stream.next(1)
     out = torch.zeros((w.batch, w.q_heads, w.head_dim), dtype=torch.float32, device=dev)
@@ -315,8 +370,11 @@ def test_a_wait_that_runs_out_ends_the_step_with_a_status():
     with pytest.raises(mkv.MkvError) as e:
         ctx.status_sync()
     elapsed = time.perf_counter() - t0
-    assert e.value.code == 7                                          # MKV_ERR_TIMEOUT
-    assert 0.015 < elapsed < 1.5                                      # it waited for the limit, not for 2 s
+    if what == "lost_tile":
+        assert e.value.code == 8 and elapsed < 1.0                   # MKV_ERR_DEVICE_CHECK, at once
+    else:
+        assert e.value.code == 7                                      # MKV_ERR_TIMEOUT
+        assert 0.015 < elapsed < 1.5                                  # it waited for the limit, not for 2 s
     with pytest.raises(mkv.MkvError):
         ctx.status_sync()                                             # sticky until reset
     ctx.reset()
