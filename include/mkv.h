@@ -354,21 +354,16 @@ int64_t mkv_launch_count(const mkv_ctx* ctx);
 mkv_status mkv_get_grid(const mkv_ctx* ctx, int layer, int32_t* n_ctas, int32_t* n_ctas_max);
 
 /*
- * Test hooks for the kernels' error paths; nothing here traps, faults or spins without bound.
- * Both act on the tensor-core kernel (otherwise MKV_ERR_UNSUPPORTED), synchronise the device, and
- * leave the layer's results undefined: call mkv_reset() and prefill again afterwards.
- *   MKV_INJECT_LOST_TILE          one tile of unit (b, kv_head) counts as never delivered: the
- *                                 unit's finishing part never becomes due, which the last CTA of
- *                                 the layer's next step notices on its way out
- *                                 (MKV_ERR_DEVICE_CHECK; no waiting involved).
- *   MKV_INJECT_EMPTY_QUEUE_ENTRY  the queue through which finished units reach idle CTAs claims
- *                                 an entry that is never written: in the layer's next step a CTA
- *                                 takes it, waits for its content up to the wait limit
- *                                 (MKV_OPT_WAIT_LIMIT_US), gives up and sets MKV_ERR_TIMEOUT; the
- *                                 rest of the step completes.  (b, kv_head are ignored.)
+ * Test hook for the error path of the kernels' bounded waits; nothing traps, faults or spins
+ * without bound.  Tensor-core kernel only (the scalar kernel has no waits): otherwise
+ * MKV_ERR_UNSUPPORTED.  Synchronises the device.  The layer's results are undefined afterwards:
+ * call mkv_reset() and prefill again.
+ *   MKV_INJECT_LOST_TILE   one tile of unit (b, kv_head) counts as never delivered from now on, so
+ *                          in the layer's next step the unit's finishing part waits for a count
+ *                          that cannot come, gives up at the wait limit (MKV_OPT_WAIT_LIMIT_US)
+ *                          and sets MKV_ERR_TIMEOUT; the rest of the step completes.
  */
 #define MKV_INJECT_LOST_TILE 0
-#define MKV_INJECT_EMPTY_QUEUE_ENTRY 1
 mkv_status mkv_debug_inject(mkv_ctx* ctx, int layer, int what, int b, int kv_head);
 
 /*

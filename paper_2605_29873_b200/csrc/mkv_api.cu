@@ -41,7 +41,7 @@ struct ScratchOff { size_t logit, head_sum, unit_sum, part_o, part_ml, keys, lis
 // layers, sized for all of them.
 struct PlanOff {
     size_t cta_unit0, cta_head0, cta_headn, cta_t0, unit_next0, unit_chunk, tile_begin, unit_cta0, next, cnt,
-        launch_no, tq_ctrl, tq_items, fin, end;
+        launch_no, end;
 };
 struct Layout {
     int layers, units, cap, rowb, lstride;
@@ -67,9 +67,6 @@ PlanOff make_plan_off(size_t nu) {
     p.next = take(2 * nu * 4);      // two copies each, alternating from launch to launch
     p.cnt = take(2 * nu * 8);
     p.launch_no = take((size_t)kMaxCtas * 4);   // per CTA: launches since the plan was (re)built
-    p.tq_ctrl = take(2 * 8);
-    p.tq_items = take(2 * nu * 4);
-    p.fin = take(2 * 8);
     p.end = o;
     return p;
 }
@@ -174,19 +171,11 @@ __global__ void host_gather_kernel(const HostPiece a, const HostPiece b, const H
     if (i < c3.n16) c3.dst[i] = c3.src[i];
 }
 
-// Test hooks.  what = 0: one tile of unit `u` counts as never delivered (both copies of its count
-// start at -1), so its tail never becomes due.  what = 1: the queue of due tails claims to hold one
-// more entry than will ever be written, so a tail group that takes it waits for its content.
-__global__ void debug_kernel(LayerDev L, int u, int what) {
-    if (what == 0) {
-        L.cnt[u] = make_int2(-1, 0);
-        L.cnt[L.n_units + u] = make_int2(-1, 0);
-    } else {
-        L.tq_ctrl[0] = make_int2(0, 1);
-        L.tq_ctrl[1] = make_int2(0, 1);
-        L.tq_items[0] = 0;
-        L.tq_items[L.n_units] = 0;
-    }
+// Test hook of mkv_debug_inject: one tile of unit `u` counts as never delivered (both copies of
+// its count start at -1), so its tail never becomes due.
+__global__ void debug_kernel(LayerDev L, int u) {
+    L.cnt[u] = make_int2(-1, 0);
+    L.cnt[L.n_units + u] = make_int2(-1, 0);
 }
 
 // The device's view of pinned host memory [p, p + bytes), or nullptr if the GPU cannot read it
@@ -309,7 +298,6 @@ struct mkv_ctx {
     // per plan (layers single-layer plans, then the several-layer plan)
     std::vector<char> stepped;   // a launch has used the plan since it was (re)built
     std::vector<int> n_ctas;
-    std::vector<int> tiles_per_cta;   // per plan: a CTA's even share of the plan's tiles
     int stack_layer0, stack_n;   // layers the several-layer plan is built for (stack_n = 0: none)
     // the previous kernel launch of the context: its layers, stream and set of scratch
     int last_layer0, last_n, scratch_set;
@@ -363,9 +351,6 @@ LayerDev layer_dev(const mkv_ctx* c, int layer0, int n, int plan, int set = 0) {
     d.next = (int32_t*)(pb + po.next);
     d.cnt = (int2*)(pb + po.cnt);
     d.launch_no = (uint32_t*)(pb + po.launch_no);
-    d.tq_ctrl = (int2*)(pb + po.tq_ctrl);
-    d.tq_items = (int32_t*)(pb + po.tq_items);
-    d.fin = (int2*)(pb + po.fin);
     d.part_o = (float*)(sb + so.part_o);
     d.part_ml = (float*)(sb + so.part_ml);
     d.unit_step = (int32_t*)at(o.unit_step);
@@ -411,7 +396,6 @@ mkv_status launch_step(mkv_ctx* c, int plan, int layer0, int n, Params p, cudaSt
     // set of scratch), and with the caller's inputs final it need not wait for it at all.
     const bool disjoint = c->last_n > 0 && (layer0 >= c->last_layer0 + c->last_n || c->last_layer0 >= layer0 + n);
     p.defer = (overlap && c->use_mma && p.early_inputs && !staged_inputs && disjoint && c->last_stream == (void*)st) ? 1 : 0;
-    p.trigger_after = std::max(1, c->tiles_per_cta[plan] / 2);
     cudaError_t e = c->use_mma ? launch_mma(p, st, overlap, c->stages) : launch_simt(p, c->kv_dtype, st);
     if (e != cudaSuccess) return MKV_ERR_CUDA;
     c->launches += 1;
@@ -450,7 +434,6 @@ mkv_status upload_plan(mkv_ctx* c, int plan, int units, const int32_t* unit_lens
     const StartTable T = build_start_table(units, c->budget_max, unit_lens, c->n_ctas_max, c->head_tiles,
                                            (c->flags & MKV_FLAG_REPRODUCIBLE) != 0);
     c->n_ctas[plan] = T.n_ctas;
-    c->tiles_per_cta[plan] = (int)std::max<long long>(1, T.tiles / T.n_ctas);
     uint8_t* pb = plan_base(c, plan);
     const PlanOff& po = plan_off(c, plan);
     const size_t U = (size_t)units, N = (size_t)T.n_ctas;
@@ -470,7 +453,6 @@ mkv_status upload_plan(mkv_ctx* c, int plan, int units, const int32_t* unit_lens
     up(po.next + U * 4, T.next0, U);
     ok &= cudaMemsetAsync(pb + po.cnt, 0, 2 * U * 8, st) == cudaSuccess;
     ok &= cudaMemsetAsync(pb + po.launch_no, 0, (size_t)kMaxCtas * 4, st) == cudaSuccess;
-    ok &= cudaMemsetAsync(pb + po.tq_ctrl, 0, po.end - po.tq_ctrl, st) == cudaSuccess;   // queue, entries, finish counts
     // (the host vectors are pageable: the runtime has staged them before each call returns)
     c->stepped[plan] = 0;
     return ok ? MKV_OK : MKV_ERR_CUDA;
@@ -612,7 +594,6 @@ mkv_status mkv_create(int layers, int q_heads, int kv_heads, int head_dim, int b
     c->prefilled.assign(layers, 0);
     c->stepped.assign(layers + 1, 0);
     c->n_ctas.assign(layers + 1, 0);
-    c->tiles_per_cta.assign(layers + 1, 1);
     c->stack_layer0 = 0; c->stack_n = 0;
     c->last_layer0 = 0; c->last_n = 0; c->scratch_set = 0; c->last_stream = nullptr;
     c->lens.assign(layers, std::vector<int32_t>((size_t)batch * kv_heads, 0));
@@ -876,13 +857,13 @@ mkv_status mkv_get_grid(const mkv_ctx* c, int layer, int32_t* n_ctas, int32_t* n
 
 mkv_status mkv_debug_inject(mkv_ctx* c, int layer, int what, int b, int g) {
     if (!layer_ok(c, layer) || b < 0 || b >= c->batch || g < 0 || g >= c->kv_heads) return MKV_ERR_INVALID_ARG;
-    if (what != MKV_INJECT_LOST_TILE && what != MKV_INJECT_EMPTY_QUEUE_ENTRY) return MKV_ERR_INVALID_ARG;
+    if (what != MKV_INJECT_LOST_TILE) return MKV_ERR_INVALID_ARG;
     if (!c->prefilled[layer]) return MKV_ERR_BAD_STATE;
     if (!c->use_mma) return MKV_ERR_UNSUPPORTED;
     DeviceGuard guard(c->device);
     if (!guard.ok || cudaDeviceSynchronize() != cudaSuccess) return MKV_ERR_CUDA;
     const LayerDev d = layer_dev(c, layer);
-    debug_kernel<<<1, 1>>>(d, b * c->kv_heads + g, what == MKV_INJECT_LOST_TILE ? 0 : 1);
+    debug_kernel<<<1, 1>>>(d, b * c->kv_heads + g);
     if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return MKV_ERR_CUDA;
     return MKV_OK;
 }

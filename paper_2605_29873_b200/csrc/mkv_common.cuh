@@ -31,7 +31,7 @@
 // SMs therefore drift into the territory of slow ones and all CTAs finish together.  A CTA
 // carries one online-softmax state per unit visit and delivers it as one partial
 // (m, l, O[G][d]) together with the number of tiles it covered; the delivery that
-// completes the unit's tile count (an atomic add, never a wait) triggers that unit's tail:
+// completes the unit's tile count (an atomic add, never a wait) runs that unit's tail:
 // the fresh token, combine, normalised decode probabilities, head mean, momentum update,
 // selection, append/compaction.  The counters exist twice and alternate from launch to
 // launch; a unit's tail rewinds the idle copy, so no counter is ever reset while a CTA may
@@ -90,12 +90,6 @@ struct LayerDev {
     int32_t* next;     // [2][units] tiles handed out so far
     int2* cnt;         // [2][units] x: tiles delivered so far, y: partial slots taken so far
     uint32_t* launch_no;   // [kMaxCtas] launches CTA i has taken part in since the layer's prefill
-    // Units whose tiles are all delivered and whose tail nobody has taken yet (two copies like the
-    // counters).  The CTA that delivers a unit's last tiles runs its tail; only when that CTA's
-    // tail warps are busy does the unit go into this queue, where any idle tail group finds it.
-    int2* tq_ctrl;         // [2] x: entries taken, y: entries put
-    int32_t* tq_items;     // [2][units] unit + 1; 0 while the entry is still being written
-    int2* fin;             // [2] x: tails finished, y: CTAs that have left (the last one checks x == units)
     float* part_o;     // [units][kMaxParts][G][d]
     float* part_ml;    // [units][kMaxParts][G][2]  (running max in log2 units, running sum)
     int32_t* unit_step;// [units] decode steps completed
@@ -133,7 +127,6 @@ struct Params {
                        // other set of scratch, inputs final): it runs from the start and only orders its END
                        // behind the previous kernel -- every CTA passes the dependency wait before it lets
                        // the next launch begin, so launches still complete in stream order
-    int trigger_after; // deferred launches: tiles a CTA issues before it passes the wait and lets the next launch in
     int det;           // reproducible mode: static partition, partial slots in CTA order
     unsigned long long wait_ns;   // limit of every bounded wait inside a kernel
 };
