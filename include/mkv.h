@@ -125,7 +125,7 @@ typedef enum {
                                   occupancy that results (4 or more stages leave room for one
                                   CTA per SM instead of two).  Layers must be prefilled again. */
     MKV_OPT_HEAD_TILES = 2,    /* 64-row prompt tiles a CTA owns outright where it starts, 0..16
-                                  (default 4): they are fetched, and with MKV_FLAG_INPUTS_READY
+                                  (default 3): they are fetched, and with MKV_FLAG_INPUTS_READY
                                   also attended, before the previous step has ended.  Layers
                                   must be prefilled again.                                    */
     MKV_OPT_WAIT_LIMIT_US = 3, /* limit of every wait inside a kernel, microseconds
@@ -157,7 +157,7 @@ size_t mkv_workspace_bytes(int layers, int batch, int q_heads, int kv_heads, int
  *   prefill_lens    host, [batch]
  *   n_ctas_max      upper bound of the grid (1..2048)
  *   n_ctas          host out: CTAs used
- *   head_tiles      tiles a CTA reserves where it starts (0..16; the library's default is 4)
+ *   head_tiles      tiles a CTA reserves where it starts (0..16; the library's default is 3)
  *   cta_unit0/head0/headn   host out, [n_ctas_max]: unit a CTA starts in, its first reserved
  *                   tile there, and how many tiles it has reserved (0 or head_tiles)
  *   unit_next0      host out, [batch*kv_heads]: reserved tiles per unit = start value of the

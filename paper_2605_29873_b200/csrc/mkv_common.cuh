@@ -51,7 +51,7 @@ constexpr int kTileRows = 64;       // rows of one tile of the work decompositio
 constexpr int kMaxGroup = 8;        // G = q_heads / kv_heads the kernels are built for
 constexpr int kMaxParts = 64;       // partials per unit (chunks grow to keep this)
 constexpr int kMaxCtas = 2048;      // persistent grid upper bound
-constexpr int kHeadTiles = 4;       // tiles a CTA owns outright at its starting place, by default
+constexpr int kHeadTiles = 3;       // tiles a CTA owns outright at its starting place, by default (the ring's depth)
 constexpr int kMaxHeadTiles = 16;   // ... and the most a context may ask for
 constexpr int kHopWindow = 256;     // units a CTA looks at, ahead of its own, when its unit runs dry
 constexpr int kMaxHome = 32;        // CTAs that start in one unit (bound kept by the start table)

@@ -141,7 +141,7 @@ def plan_ranges(batch, kv_heads, budget, prefill_lens, n_ctas_max):
     return t0[: n.value + 1].copy(), tb, uc
 
 
-def plan_starts(batch, kv_heads, budget, prefill_lens, n_ctas_max, head_tiles=4):
+def plan_starts(batch, kv_heads, budget, prefill_lens, n_ctas_max, head_tiles=3):
     """The kernels' start table for these lengths (``mkv_plan_starts``; host arithmetic only).
     Returns (cta_unit0, cta_head0, cta_headn, unit_next0, unit_chunk) as int32 arrays."""
     lens = np.ascontiguousarray(prefill_lens, dtype=np.int32)

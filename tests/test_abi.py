@@ -109,7 +109,7 @@ def test_start_table_invariants(lib):
         for c in range(len(u0)):
             t0 = tiles.sum() * c // len(u0)
             assert begin[u0[c]] <= t0 < begin[u0[c] + 1]
-        assert set(hn.tolist()) <= {0, 4}
+        assert set(hn.tolist()) <= {0, 3}
         # another reservation size: same spread, reserved ranges of that size
         u0b, h0b, hnb, nxb, _ = mkv.plan_starts(B, hkv, budget, lens, nmax, head_tiles=7)
         assert (u0b == u0).all() and set(hnb.tolist()) <= {0, 7} and (nxb % 7 == 0).all()
@@ -118,8 +118,8 @@ def test_start_table_invariants(lib):
             mine = np.where(u0 == u)[0]
             got = sorted((int(h0[c]), int(hn[c])) for c in mine if hn[c] > 0)
             # reserved ranges tile [0, next0) without gaps, all inside the prefill tiles
-            assert [g[0] for g in got] == list(range(0, 4 * len(got), 4))
-            assert nx[u] == 4 * len(got) <= -(-int(lens[u // hkv]) // 64)
+            assert [g[0] for g in got] == list(range(0, 3 * len(got), 3))
+            assert nx[u] == 3 * len(got) <= -(-int(lens[u // hkv]) // 64)
             assert len(mine) <= 32 and ch[u] >= 2
             assert len(mine) + -(-int(tiles[u] - nx[u]) // int(ch[u])) <= 64 - 8
 
