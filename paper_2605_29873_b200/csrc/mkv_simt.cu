@@ -210,14 +210,20 @@ __global__ void __launch_bounds__(kSimtThreads) simt_kernel(const Params p) {
         }
         // ---- next unit (cyclically after this one) that still has tiles to hand out -----------
         if (det) { ++u; if (u >= U) break; continue; }
-        if (tid == 0) {
+        if (warp == 0) {     // 32 candidates per trip, the nearest one with tiles left wins
             int found = -1;
-            for (int k = 1; k < U && k <= kHopWindow; ++k) {
-                const int cand = (u + k) % U;
-                const int nd = min(L.n_dec[cand], p.cap - (dec ? 1 : 0));
-                if (__ldcg(&nxt[cand]) < unit_tiles(L.unit_lp[cand], nd)) { found = cand; break; }
+            for (int base = 1; base < U && base <= kHopWindow && found < 0; base += 32) {
+                const int k = base + lane;
+                bool has = false;
+                if (k < U) {
+                    const int cand = (u + k) % U;
+                    const int nd = min(L.n_dec[cand], p.cap - (dec ? 1 : 0));
+                    has = __ldcg(&nxt[cand]) < unit_tiles(L.unit_lp[cand], nd);
+                }
+                const unsigned m = __ballot_sync(0xffffffffu, has);
+                if (m) found = (u + base + __ffs(m) - 1) % U;
             }
-            s_u = found;
+            if (lane == 0) s_u = found;
         }
         __syncthreads();
         u = s_u;

@@ -1,6 +1,6 @@
 """The multi-GPU path of bench.py without GPUs: two gloo ranks on the CPU run the pieces that
-differ from the single-rank run -- per-rank workloads, the max-over-ranks timing reduction and
-the whole-job throughput -- and the oracle confirms that ranks really hold independent data."""
+differ from the single-rank run -- per-rank workloads (different seeds, hence different data),
+the max-over-ranks timing reduction and the whole-job throughput."""
 import os
 import sys
 
