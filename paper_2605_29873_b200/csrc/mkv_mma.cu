@@ -29,7 +29,8 @@
 //     ring stage borrowed from the producer and go straight on to the next unit; the merge
 //     warp folds the four states into one partial in global memory, returns the stage, adds
 //     the visit's tiles to the unit's count.
-//   * four TAIL warps, which watch the counts of the units assigned to this CTA and run a
+//   * four TAIL warps, which watch the counts of the units this CTA looks after (the ones it starts
+//     in) and run a
 //     unit's tail (fresh token, combine, probabilities, momentum update, selection,
 //     append/compaction) as soon as its count is complete, while the stream continues.
 //     (Handing a completed unit to the CTA that delivered its last tiles instead, with a queue
@@ -159,7 +160,17 @@ __device__ void tail_group(const Params& p, Control* ctl, TailSmem<kTailThreads>
         ptx::griddep_launch_dependents();
         MKV_TR(7);
     }
-    for (int u = blockIdx.x; u < L.n_units; u += gridDim.x) {
+    // Which units this CTA looks after: the unit it starts in, if it is the first CTA to start
+    // there, and the units after it in which no CTA starts, if it is the last one to start there.
+    // Those are the units it streams first, in this order, so they also complete in this order
+    // (a launch over many layers has more units than CTAs).
+    const int c = (int)blockIdx.x;
+    const int u_first = L.cta_unit0[c];
+    const bool first_there = (c == 0) || (L.cta_unit0[c - 1] != u_first);
+    const bool last_there = (c + 1 == (int)gridDim.x) || (L.cta_unit0[c + 1] != u_first);
+    const int u_begin = first_there ? u_first : u_first + 1;
+    const int u_end = last_there ? ((c + 1 == (int)gridDim.x) ? L.n_units : L.cta_unit0[c + 1]) : u_first + 1;
+    for (int u = u_begin; u < u_end; ++u) {
         TailPre<kTailThreads, GB> pre;
         tail_prefetch<__nv_bfloat16, kTailThreads, GB, LAYER>(p, u, *tsm, tt, pre);
         if (tt == 0) {
