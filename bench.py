@@ -293,7 +293,7 @@ class Arm:
     """One configuration set up on the device at steady state: context, input ring, step functions."""
 
     def __init__(self, torch, mkv, w, lens, layers, dev, seed, inputs, score_mode="group", kernel="auto", stacked=False,
-                 out_dtype=None, head_tiles=None, fill=None, early=True):
+                 out_dtype=None, head_tiles=None, fill=None, early=True, grid_share=None):
         self.torch, self.w, self.layers, self.stacked = torch, w, layers, stacked
         B, Hq, Hkv, d = w.batch, w.q_heads, w.kv_heads, w.head_dim
         kv_dtype = mkv.MKV_BF16 if w.dtype == "bf16" else mkv.MKV_F32
@@ -307,6 +307,8 @@ class Arm:
                                 flags=mkv.MKV_FLAG_INPUTS_READY if early else 0)
         if head_tiles is not None:
             self.ctx.set_option(mkv.MKV_OPT_HEAD_TILES, head_tiles)
+        if grid_share is not None:
+            self.ctx.set_option(mkv.MKV_OPT_GRID_SHARE, grid_share)
         gen = torch.Generator(device=dev)
         gen.manual_seed(seed)
         for layer in range(layers):
@@ -431,6 +433,7 @@ def main():
     ap.add_argument("--budget", type=int, default=0, help="override the workload's decode budget (profiling small cases)")
     ap.add_argument("--inputs", default="hot", choices=["hot", "plain"], help="kind of device-generated step inputs")
     ap.add_argument("--head-tiles", type=int, default=-1, help="reserved prompt tiles per CTA (default: the library's)")
+    ap.add_argument("--grid-share", type=int, default=-1, help="percent of the resident CTA slots a step uses (default: the library's)")
     ap.add_argument("--no-early", action="store_true", help="do not promise that the inputs are final at enqueue time")
     ap.add_argument("--per-layer", action="store_true", help="llama_stack: one launch per layer instead of one per stack")
     ap.add_argument("--rounds", type=int, default=5)
@@ -478,8 +481,10 @@ def main():
     tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
     head_tiles = args.head_tiles if args.head_tiles >= 0 else None
     arm = Arm(torch, mkv, w, lens, args.layers, dev, 1234 + rank, args.inputs, score_mode=args.score_mode,
-              kernel=args.kernel, stacked=stacked, head_tiles=head_tiles, early=not args.no_early)
+              kernel=args.kernel, stacked=stacked, head_tiles=head_tiles, early=not args.no_early,
+              grid_share=args.grid_share if args.grid_share > 0 else None)
     ctx = arm.ctx
+    ctx_grid = ctx.grid(0)
     stream = torch.cuda.current_stream(dev)
     # The ramp: every layer's decode pool from empty to the budget, timed on its own (steps get
     # longer as the pool grows); it also is the set-up of the steady state measured below.
@@ -572,6 +577,7 @@ def main():
         cfg = workload_config(w, lens, args, args.inputs, older)
         cfg["launch"] = (f"one launch per {arm.per_call}-layer stack" if stacked else "one launch per layer-step")
         cfg["early_inputs"] = not args.no_early
+        cfg["grid"] = "%d CTAs of %d resident" % ctx_grid
         line = {
             "metric": "decode tokens/sec per layer", "value": tokens_per_s, "unit": "tokens/s",
             "n_gpus": world, "steps": calls * arm.per_call, "warmup": args.warmup, "ms_per_step": ms_per_step,

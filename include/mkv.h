@@ -131,9 +131,17 @@ typedef enum {
     MKV_OPT_WAIT_LIMIT_US = 3, /* limit of every wait inside a kernel, microseconds
                                   (default 2,000,000); on expiry the step ends early and the
                                   sticky status becomes MKV_ERR_TIMEOUT                       */
-    MKV_OPT_OVERLAP = 4        /* 1 (default): consecutive steps on a stream overlap their
+    MKV_OPT_OVERLAP = 4,       /* 1 (default): consecutive steps on a stream overlap their
                                   start-up with the previous step's end (programmatic
                                   dependent launch); 0: plain stream order                    */
+    MKV_OPT_GRID_SHARE = 5     /* percent (10..100) of the CTAs the GPU can keep resident that a
+                                  single-layer step uses.  Default 100, and 75 with
+                                  MKV_FLAG_INPUTS_READY: steps of different layers then run side
+                                  by side, and a step that leaves a quarter of the CTA slots
+                                  free lets its successor begin streaming at once instead of
+                                  waiting for slots.  A context with that flag whose steps all
+                                  go to the same layer should set 100.  Steps over several
+                                  layers always use all slots.  Layers must be prefilled again. */
 } mkv_option;
 
 /*

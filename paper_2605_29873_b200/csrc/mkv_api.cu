@@ -235,7 +235,16 @@ StartTable build_start_table(int units, int budget, const int32_t* unit_lens, in
     for (int u = 0; u < U; ++u) t_max = std::max(t_max, tile_begin[u + 1] - tile_begin[u]);
     // a unit of t tiles draws at most ceil(n_ctas * t / t_all) CTAs: keep that within kMaxHome
     const long long home_cap = (long long)(kMaxHome - 1) * t_all / t_max;
-    const int n_ctas = (int)std::max<long long>(1, std::min<long long>(std::min<long long>(n_ctas_max, t_all / 2), home_cap));
+    int n_ctas = (int)std::max<long long>(1, std::min<long long>(std::min<long long>(n_ctas_max, t_all / 2), home_cap));
+    // Units of equal size (a batch of equal prompts): make CTA stretches and units line up -- a
+    // whole number of CTAs per unit, or a whole number of units per CTA -- so that no unit is
+    // shared by CTAs that also serve its neighbours and most units end up with a single partial.
+    bool equal = U > 1;
+    for (int u2 = 1; u2 < U && equal; ++u2) equal = (tile_begin[u2 + 1] - tile_begin[u2]) == tile_begin[1];
+    if (equal && !det) {
+        if (n_ctas >= U) n_ctas = n_ctas / U * U;
+        else n_ctas = ceil_div(U, ceil_div(U, n_ctas));
+    }
     T.n_ctas = n_ctas;
     T.tiles = t_all;
     T.cta_unit0.assign(n_ctas, 0);
@@ -292,6 +301,7 @@ struct mkv_ctx {
     bool use_mma;
     int stages;     // ring depth of the tensor-core kernel
     int head_tiles; // tiles a CTA owns outright at its starting place
+    int grid_share; // percent of n_ctas_max that a single-layer launch uses
     bool pdl;       // consecutive launches overlap (programmatic dependent launch)
     unsigned long long wait_ns;
     std::vector<char> prefilled;
@@ -431,7 +441,11 @@ mkv_status size_grid(mkv_ctx* c) {
 
 // Writes a plan (start table, fresh counters) for `units` units with the given prompt lengths.
 mkv_status upload_plan(mkv_ctx* c, int plan, int units, const int32_t* unit_lens, cudaStream_t st) {
-    const StartTable T = build_start_table(units, c->budget_max, unit_lens, c->n_ctas_max, c->head_tiles,
+    // Launches of one layer leave part of the SMs' CTA slots to the launch that runs alongside
+    // (the next layer's, see Params::defer); a launch over several layers is never followed by
+    // one that could, and takes them all.
+    const int n_max = plan < c->layers ? std::max(1, (int)((long long)c->n_ctas_max * c->grid_share / 100)) : c->n_ctas_max;
+    const StartTable T = build_start_table(units, c->budget_max, unit_lens, n_max, c->head_tiles,
                                            (c->flags & MKV_FLAG_REPRODUCIBLE) != 0);
     c->n_ctas[plan] = T.n_ctas;
     uint8_t* pb = plan_base(c, plan);
@@ -581,6 +595,7 @@ mkv_status mkv_create(int layers, int q_heads, int kv_heads, int head_dim, int b
     c->use_mma = use_mma;
     c->stages = 3;
     c->head_tiles = kHeadTiles;
+    c->grid_share = (flags & MKV_FLAG_INPUTS_READY) ? 75 : 100;
     c->pdl = true;
     c->wait_ns = 2000000000ull;   // 2 s
     const mkv_status gs = size_grid(c);
@@ -621,6 +636,10 @@ mkv_status mkv_set_option(mkv_ctx* c, int option, long long value) {
         case MKV_OPT_HEAD_TILES:
             if (value < 0 || value > kMaxHeadTiles) return MKV_ERR_INVALID_ARG;
             c->head_tiles = (int)value;
+            break;
+        case MKV_OPT_GRID_SHARE:
+            if (value < 10 || value > 100) return MKV_ERR_INVALID_ARG;
+            c->grid_share = (int)value;
             break;
         case MKV_OPT_WAIT_LIMIT_US:
             if (value < 1 || value > 60000000ll) return MKV_ERR_INVALID_ARG;

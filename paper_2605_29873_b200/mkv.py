@@ -13,7 +13,7 @@ MKV_BF16, MKV_F32 = 0, 1
 MKV_SCORE_GROUP_MEAN, MKV_SCORE_LAYER_MEAN = 0, 1
 MKV_KERNEL_AUTO, MKV_KERNEL_SIMT, MKV_KERNEL_MMA = 0, 1, 2
 MKV_FLAG_RECORD_PROBS, MKV_FLAG_INPUTS_READY, MKV_FLAG_REPRODUCIBLE = 1, 2, 4
-MKV_OPT_RING_STAGES, MKV_OPT_HEAD_TILES, MKV_OPT_WAIT_LIMIT_US, MKV_OPT_OVERLAP = 1, 2, 3, 4
+MKV_OPT_RING_STAGES, MKV_OPT_HEAD_TILES, MKV_OPT_WAIT_LIMIT_US, MKV_OPT_OVERLAP, MKV_OPT_GRID_SHARE = 1, 2, 3, 4, 5
 MKV_INJECT_LOST_TILE = 0
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
