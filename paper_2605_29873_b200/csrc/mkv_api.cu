@@ -196,7 +196,6 @@ constexpr int kMinChunk = 2;   // tiles per pull of a unit's counter, lower boun
 
 struct StartTable {
     int n_ctas = 0;
-    long long tiles = 0;      // all units' tiles with full decode pools
     std::vector<int32_t> lp, next0, chunk, cta_unit0, cta_head0, cta_headn;
     // reproducible mode
     std::vector<int32_t> tile_begin, cta_t0, unit_cta0;
@@ -246,7 +245,6 @@ StartTable build_start_table(int units, int budget, const int32_t* unit_lens, in
         else n_ctas = ceil_div(U, ceil_div(U, n_ctas));
     }
     T.n_ctas = n_ctas;
-    T.tiles = t_all;
     T.cta_unit0.assign(n_ctas, 0);
     T.cta_head0.assign(n_ctas, 0);
     T.cta_headn.assign(n_ctas, 0);
