@@ -358,7 +358,9 @@ mkv_status mkv_attend_noalloc(const void* q, const void* K, const void* V, void*
 /* Number of kernels this context has launched so far (host counter). */
 int64_t mkv_launch_count(const mkv_ctx* ctx);
 
-/* The grid of `layer`'s launches (0 before its prefill) and the bound it was sized under. */
+/* The grid of `layer`'s launches (0 before its prefill) and the number of CTAs the GPU keeps
+ * resident, which bounds every grid.  layer == the context's layer count asks for the grid of
+ * the launches over several layers (0 before the first such launch). */
 mkv_status mkv_get_grid(const mkv_ctx* ctx, int layer, int32_t* n_ctas, int32_t* n_ctas_max);
 
 /*

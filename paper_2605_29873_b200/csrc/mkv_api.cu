@@ -866,8 +866,9 @@ mkv_status mkv_status_sync(mkv_ctx* c, void* stream) {
 int64_t mkv_launch_count(const mkv_ctx* c) { return c ? c->launches : 0; }
 
 mkv_status mkv_get_grid(const mkv_ctx* c, int layer, int32_t* n_ctas, int32_t* n_ctas_max) {
-    if (!layer_ok(c, layer) || !n_ctas || !n_ctas_max) return MKV_ERR_INVALID_ARG;
-    *n_ctas = c->prefilled[layer] ? c->n_ctas[layer] : 0;
+    if (!c || layer < 0 || layer > c->layers || !n_ctas || !n_ctas_max) return MKV_ERR_INVALID_ARG;
+    if (layer == c->layers) *n_ctas = c->stack_n > 0 ? c->n_ctas[layer] : 0;
+    else *n_ctas = c->prefilled[layer] ? c->n_ctas[layer] : 0;
     *n_ctas_max = c->n_ctas_max;
     return MKV_OK;
 }
