@@ -315,6 +315,55 @@ def test_reproducible_mode_gives_the_same_bits_twice(case):
         c.close()
 
 
+def test_reproducible_mode_with_launches_side_by_side():
+    """Both flags together: launches on different layers overlap in time, but each has its own
+    scratch and a fixed partition, so two contexts stepped the same way still agree bit for bit
+    (outputs of every step, pools and scores of both layers at the end)."""
+    import torch
+    w = CONFIGS["llama_b16"].with_(batch=4, prefill=(200, 1500), steps=80, budget=48, variant="hot", n_heavy=2)
+    n_layers = 2
+    ws = [w.with_(seed=70 + l) for l in range(n_layers)]
+    max_pre = max(int(x.prefill_lens().max()) for x in ws)
+    flags = mkv.MKV_FLAG_REPRODUCIBLE | mkv.MKV_FLAG_INPUTS_READY
+    ctxs = [mkv.MomentKV(n_layers, w.q_heads, w.kv_heads, w.head_dim, w.budget, w.beta, w.batch, max_pre,
+                         out_dtype=mkv.MKV_F32, flags=flags) for _ in range(2)]
+    streams = [BatchStream(ws[l], l) for l in range(n_layers)]
+    oracles = [prefill_both(ctxs[0], ws[l], streams[l], layer=l)[0] for l in range(n_layers)]
+    for l in range(n_layers):
+        prefill_both(ctxs[1], ws[l], BatchStream(ws[l], l), layer=l)
+    dt, dev = ctxs[0].torch_kv_dtype(), ctxs[0].device
+    burst = 20
+    outs = [torch.zeros((burst, n_layers, w.batch, w.q_heads, w.head_dim), dtype=torch.float32, device=dev) for _ in range(2)]
+    for start in range(0, w.steps, burst):
+        (qs, ks, vs), (qd, kd, vd) = stacked_inputs(streams, burst, torch, dt, dev)
+        torch.cuda.synchronize()
+        for c in range(2):
+            for j in range(burst):
+                for l in range(n_layers):
+                    ctxs[c].decode_step(l, qd[j, l], kd[j, l], vd[j, l], outs[c][j, l])
+            ctxs[c].status_sync()
+        assert torch.equal(outs[0], outs[1]), f"steps {start}..: outputs differ between two runs"
+        got = outs[0].double().cpu().numpy()
+        for j in range(burst):
+            for l in range(n_layers):
+                for b in range(w.batch):
+                    ref = oracles[l][b].attend_update(qs[j, l, b], ks[j, l, b], vs[j, l, b])
+                    rowmax = np.abs(ref).max(axis=1)
+                    assert (np.abs(got[j, l, b] - ref).max(axis=1) <= 2e-3 * rowmax).all(), (start + j, l, b)
+                    oracles[l][b].evict()
+    for l in range(n_layers):
+        for b in range(w.batch):
+            for g in range(w.kv_heads):
+                (p0, s0), (p1, s1) = (c.decode_state(l, b, g) for c in ctxs)
+                np.testing.assert_array_equal(p0, p1)
+                np.testing.assert_array_equal(s0.view(np.uint32), s1.view(np.uint32))
+                (K0, V0), (K1, V1) = (c.read_kv(l, b, g, 1) for c in ctxs)
+                np.testing.assert_array_equal(K0, K1)
+                np.testing.assert_array_equal(V0, V1)
+    for c in ctxs:
+        c.close()
+
+
 @pytest.mark.parametrize("stages", [2, 5])
 def test_ring_depth_resizes_the_grid(stages):
     """MKV_OPT_RING_STAGES: with five 32 KB stages only one CTA of the tensor-core kernel fits an
